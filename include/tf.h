@@ -1,0 +1,176 @@
+/*
+ * tf.h -- C boundary of the B200 (sm_100a) Token Filtering layer step.
+ *
+ * One attention layer of a prefill sequence, as the paper's Algorithm 1 defines it
+ * for "the current token", applied to every token t with tokens 0..t-1 as its past:
+ *
+ *   tf_kv_stats          anchors (running mean of past K / V per head) and the per-head
+ *                        cosine similarity of each token's K and V to them
+ *   tf_score_fuse        mean / variance over heads, variance-aware weight (Eq. 2) and
+ *                        fused score S_KV (Eq. 3), one per token
+ *   tf_select            which tokens skip attention at the target pruning ratio (or
+ *                        above a threshold, Alg. 1 "skip if s_KV > tau"), compacted
+ *   tf_pruned_attention  causal attention for retained tokens only; skipped tokens'
+ *                        output rows are zero (Section 3.2)
+ *   tf_layer_filter      the four steps chained on one stream
+ *
+ * Conventions, unless an argument says otherwise:
+ *   - every tensor pointer is DEVICE memory owned by the caller; the library reads its
+ *     inputs, writes its outputs, keeps no pointer after the call returns;
+ *   - calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*,
+ *     NULL = default stream), do not synchronise and do not allocate;
+ *   - the return value reports host-side validation and launch errors only; conditions
+ *     found on the device (a bounded wait that gave up) are read with tf_get_status;
+ *   - head_dim must be 128; Q/K/V/O rows (head_dim elements) are contiguous and 16-byte
+ *     aligned, every stride a multiple of 8 elements (bf16) / 4 elements (fp32).
+ */
+#ifndef TF_H_
+#define TF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tf_ctx tf_ctx; /* opaque: device id, device status word, workspace binding */
+
+typedef enum {
+    TF_OK = 0,
+    TF_ERR_INVALID_ARG = 1, /* NULL required pointer, bad enum, ratio outside [0,1), ... */
+    TF_ERR_UNSUPPORTED = 2, /* head_dim != 128, dtype unknown, misaligned stride          */
+    TF_ERR_WORKSPACE = 3,   /* no workspace bound, or too small for this shape            */
+    TF_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                        */
+    TF_ERR_TIMEOUT = 5,     /* device: a bounded wait inside a kernel gave up             */
+    TF_ERR_NAN_SCORE = 6    /* device: a NaN score was seen (it is never pruned)          */
+} tf_status;
+
+typedef enum { TF_F32 = 0, TF_BF16 = 1 } tf_dtype;
+
+/* anchor_mode: what "mean of previous keys" (Section 3.2 / Alg. 1) covers */
+enum { TF_ANCHOR_PAST_MEAN = 0, /* tokens strictly before t (default)                     */
+       TF_ANCHOR_INCL_MEAN = 1, /* tokens up to and including t (Alg. 1 read literally)   */
+       TF_ANCHOR_EMA = 2 };     /* Eq. 1: anchor <- gamma*anchor + (1-gamma)*x, compare first */
+/* fuse_mode: the weight alpha of Eq. 2-3 */
+enum { TF_FUSE_INVVAR = 0,      /* alpha = var_v/(var_k+var_v): lower variance weighs more */
+       TF_FUSE_EQ2_LITERAL = 1, /* alpha = var_k/(var_k+var_v): Eq. 2 exactly as printed   */
+       TF_FUSE_KEY_ONLY = 2, TF_FUSE_VALUE_ONLY = 3, /* criterion ablation (Section 4.4)   */
+       TF_FUSE_MEAN = 4 };      /* alpha = 1/2 (Figure 1 caption)                          */
+enum { TF_SELECT_RATIO = 0,     /* prune exactly P = min(E, floor(ratio*S)) top-scoring eligible tokens */
+       TF_SELECT_THRESHOLD = 1 }; /* prune eligible tokens with score > threshold (strict) */
+enum { TF_KV_ALL = 0,           /* retained queries see every earlier token's K/V (default) */
+       TF_KV_RETAINED = 1 };    /* retained queries see retained tokens' K/V only           */
+
+/* Problem shape.  Tensors are addressed as base + b*stride[0] + t*stride[1] + h*stride[2] + i,
+ * in ELEMENTS, i in [0, head_dim).  Query head q reads KV head q / (n_q_heads / n_kv_heads). */
+typedef struct {
+    int32_t batch, seq, n_q_heads, n_kv_heads, head_dim;
+    int32_t dtype;          /* tf_dtype of Q, K, V and O                                     */
+    int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];
+    int32_t window;         /* 0: key j visible to query t iff j <= t; W>0: also j > t - W   */
+    float softmax_scale;    /* 0 => 1/sqrt(head_dim)                                         */
+} tf_shape;
+
+/* Method parameters (Alg. 1 inputs and the readings of it that are selectable). */
+typedef struct {
+    double prune_ratio;       /* RATIO mode: target fraction of the S tokens to prune, in [0,1) */
+    int32_t warmup_tokens;    /* the first n tokens of each sequence are never pruned (Section 3.2 warm-up) */
+    const uint8_t *eligible;  /* optional device [B,S]: 1 = may be pruned; NULL = all             */
+    int32_t anchor_mode;      /* TF_ANCHOR_*                                                      */
+    float gamma;              /* EMA smoothing factor of Eq. 1 (EMA mode only)                    */
+    int32_t fuse_mode;        /* TF_FUSE_*                                                        */
+    float var_eps;            /* added to each variance so alpha is defined when both are 0; 0 => 1e-8 */
+    int32_t select_mode;      /* TF_SELECT_*                                                      */
+    const float *threshold;   /* THRESHOLD mode: device [B]                                       */
+    int32_t kv_visibility;    /* TF_KV_*                                                          */
+} tf_filter_params;
+
+/* Optional anchor state carried between calls (chunked prefill, prefill -> decode): the sums
+ * (EMA mode: the anchors) over all tokens seen so far, fp32 [B, n_kv_heads, head_dim], and the
+ * token count per sequence [B].  Any pointer may be NULL (in: no past; out: not wanted). */
+typedef struct {
+    const float *sum_k_in, *sum_v_in;
+    const int64_t *count_in;
+    float *sum_k_out, *sum_v_out;
+} tf_carry;
+
+/* Fill p with the defaults: ratio 0.5, warm-up 1 token, past-mean anchors, inverse-variance
+ * fusion, ratio selection, all K/V visible. */
+void tf_default_params(tf_filter_params *p);
+
+/* Create / destroy a context on CUDA device `device` (allocates a few words of device memory
+ * for the status record; the only allocation the library makes besides tf_layer_filter_host). */
+tf_status tf_create(tf_ctx **out, int device);
+tf_status tf_destroy(tf_ctx *ctx);
+
+/* Scratch the kernels need for this shape (scan look-back records, and the intermediates of
+ * tf_layer_filter that the caller does not ask for).  The caller allocates it (256-byte aligned
+ * device memory) and binds it; one workspace serves one call at a time. */
+tf_status tf_workspace_bytes(const tf_shape *shape, const tf_filter_params *params, size_t *bytes);
+tf_status tf_set_workspace(tf_ctx *ctx, void *device_ptr, size_t bytes);
+
+/* Steps a1+a2 (Alg. 1 lines AnchorK/AnchorV and cosine_sim; Section 3.2).  Reads K and V
+ * [B,S,n_kv_heads,128] once; writes sim_k, sim_v: contiguous fp32 [B,S,n_kv_heads], the cosine
+ * of token t's key / value to the anchor of its past (0 where there is no past; each norm is
+ * clamped at 1e-8).  carry may be NULL.  Needs the bound workspace. */
+tf_status tf_kv_stats(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                      const void *K, const void *V, float *sim_k, float *sim_v,
+                      const tf_carry *carry, void *stream);
+
+/* Step a3 (Alg. 1 lines (s_k, sigma_k^2), alpha, s_KV; Eq. 2-3).  sim_k, sim_v fp32
+ * [B,S,n_kv_heads] -> score fp32 [B,S].  Population variance over the KV heads. */
+tf_status tf_score_fuse(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                        const float *sim_k, const float *sim_v, float *score, void *stream);
+
+/* Step a4 (Alg. 1 "skip if s_KV > tau"; Section 3.3 target skip ratio; Section 3.2 warm-up).
+ * score fp32 [B,S] -> keep_mask u8 [B,S] (1 = retained), kept_idx i32 [B,S] (ascending retained
+ * positions, then -1), n_kept i32 [B], theta fp32 [B] (lowest pruned score, +inf if none;
+ * may be NULL).  RATIO mode prunes the P highest-scoring eligible tokens, equal scores resolved
+ * toward the later token; a NaN score is never pruned. */
+tf_status tf_select(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                    const float *score, uint8_t *keep_mask, int32_t *kept_idx, int32_t *n_kept,
+                    float *theta, void *stream);
+
+/* Step a5 (Section 3.2: skipped tokens' attention output is zero; standard causal softmax
+ * attention otherwise).  For every retained token kept_idx[b, i], i < n_kept[b], and query head
+ * q: O = softmax(scale * Q.K^T over visible keys) V.  Every other row of O is set to zero, so O
+ * is fully written.  kept_idx / n_kept are device arrays as tf_select writes them. */
+tf_status tf_pruned_attention(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                              const void *Q, const void *K, const void *V,
+                              const int32_t *kept_idx, const int32_t *n_kept, void *O, void *stream);
+
+/* All of Algorithm 1 for one layer plus the attention it gates: kv_stats -> score_fuse ->
+ * select -> pruned_attention on one stream.  score, keep_mask, kept_idx, n_kept are optional
+ * outputs (NULL: kept in the workspace).  Needs the bound workspace. */
+tf_status tf_layer_filter(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                          const void *Q, const void *K, const void *V, void *O,
+                          float *score, uint8_t *keep_mask, int32_t *kept_idx, int32_t *n_kept,
+                          void *stream);
+
+/* The same layer step for callers whose tensors live in HOST memory (pinned memory makes the
+ * copies asynchronous): copies Q, K, V to device staging buffers that the context owns and grows
+ * on demand (this entry point allocates; it also binds its own workspace), runs tf_layer_filter,
+ * copies O and the optional outputs back and synchronises the stream before returning.
+ * shape strides describe the host tensors; they must be dense token-major [B,S,H,128]. */
+tf_status tf_layer_filter_host(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                               const void *Q_host, const void *K_host, const void *V_host,
+                               void *O_host, float *score_host, uint8_t *keep_mask_host,
+                               int32_t *kept_idx_host, int32_t *n_kept_host, void *stream);
+
+/* Device-side conditions since the last tf_clear_status: returns TF_OK, TF_ERR_TIMEOUT or
+ * TF_ERR_NAN_SCORE.  sync != 0 synchronises the device first.  detail (may be NULL) receives
+ * four words: {code, where, count of NaN scores, kernels launched by this context}. */
+tf_status tf_get_status(tf_ctx *ctx, int sync, int64_t detail[4]);
+tf_status tf_clear_status(tf_ctx *ctx);
+
+/* Which attention kernel a bf16 call uses: 1 = tcgen05 tensor-core kernel (default),
+ * 0 = the plain CUDA-core kernel that fp32 always uses.  For A/B checks. */
+tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
+
+const char *tf_status_string(tf_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TF_H_ */

@@ -1,0 +1,200 @@
+"""ctypes binding of the C-ABI library declared in ``include/tf.h``.
+
+Argument marshalling only: every step of the layer runs in the CUDA kernels of
+``libtokenfilter.so``.  torch supplies device memory and the current stream.
+There is no fallback -- if the library is missing, loading raises.
+
+Tensors are token-major ``[B, S, H, 128]`` (any strides whose last dim is dense).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtokenfilter.so")
+
+TF_OK, TF_ERR_INVALID_ARG, TF_ERR_UNSUPPORTED, TF_ERR_WORKSPACE, TF_ERR_CUDA, TF_ERR_TIMEOUT, TF_ERR_NAN_SCORE = range(7)
+TF_F32, TF_BF16 = 0, 1
+TF_ANCHOR_PAST_MEAN, TF_ANCHOR_INCL_MEAN, TF_ANCHOR_EMA = 0, 1, 2
+TF_FUSE_INVVAR, TF_FUSE_EQ2_LITERAL, TF_FUSE_KEY_ONLY, TF_FUSE_VALUE_ONLY, TF_FUSE_MEAN = 0, 1, 2, 3, 4
+TF_SELECT_RATIO, TF_SELECT_THRESHOLD = 0, 1
+TF_KV_ALL, TF_KV_RETAINED = 0, 1
+
+EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
+           "tf_kv_stats", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
+           "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
+           "tf_status_string")
+
+
+class tf_shape(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("seq", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("dtype", C.c_int32),
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3),
+                ("v_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
+                ("window", C.c_int32), ("softmax_scale", C.c_float)]
+
+
+class tf_filter_params(C.Structure):
+    _fields_ = [("prune_ratio", C.c_double), ("warmup_tokens", C.c_int32),
+                ("eligible", C.c_void_p), ("anchor_mode", C.c_int32), ("gamma", C.c_float),
+                ("fuse_mode", C.c_int32), ("var_eps", C.c_float), ("select_mode", C.c_int32),
+                ("threshold", C.c_void_p), ("kv_visibility", C.c_int32)]
+
+
+class tf_carry(C.Structure):
+    _fields_ = [("sum_k_in", C.c_void_p), ("sum_v_in", C.c_void_p), ("count_in", C.c_void_p),
+                ("sum_k_out", C.c_void_p), ("sum_v_out", C.c_void_p)]
+
+
+class TokenFilterError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {status_string(code)} (tf_status {code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with __graft_entry__.build() "
+                               "(python -m paper_2512_07090_b200.build); there is no CPU fallback")
+        L = C.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            getattr(L, name).restype = C.c_int
+        L.tf_default_params.restype = None
+        L.tf_status_string.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().tf_status_string(C.c_int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != TF_OK:
+        raise TokenFilterError(code, what)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def default_params(**kw) -> tf_filter_params:
+    p = tf_filter_params()
+    lib().tf_default_params(C.byref(p))
+    for k, v in kw.items():
+        if k in ("eligible", "threshold"):
+            v = None if v is None else v.data_ptr()
+        setattr(p, k, v)
+    return p
+
+
+def make_shape(Q: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, O: Optional[torch.Tensor] = None,
+               window: int = 0, softmax_scale: float = 0.0, n_q_heads: Optional[int] = None) -> tf_shape:
+    """Describe ``[B,S,H,128]`` tensors (element strides of batch, token, head)."""
+    B, S, Hkv, d = K.shape
+    s = tf_shape()
+    s.batch, s.seq, s.n_kv_heads, s.head_dim = B, S, Hkv, d
+    s.n_q_heads = Q.shape[2] if Q is not None else (n_q_heads or Hkv)
+    s.dtype = {torch.float32: TF_F32, torch.bfloat16: TF_BF16}[K.dtype]
+    for name, t in (("q_stride", Q), ("k_stride", K), ("v_stride", V), ("o_stride", O if O is not None else Q)):
+        if t is None:
+            t = K
+        assert t.stride(3) == 1, "head_dim must be contiguous"
+        getattr(s, name)[:] = [t.stride(0), t.stride(1), t.stride(2)]
+    s.window, s.softmax_scale = int(window), float(softmax_scale)
+    return s
+
+
+class Context:
+    """Owns a tf_ctx and (optionally) a torch-allocated workspace bound to it."""
+
+    def __init__(self, device: int = 0):
+        self._h = C.c_void_p()
+        _check(lib().tf_create(C.byref(self._h), C.c_int(device)), "tf_create")
+        self.device = device
+        self._ws = None
+
+    def close(self):
+        if self._h:
+            lib().tf_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- workspace -----------------------------------------------------------------------------
+    def workspace_bytes(self, shape: tf_shape, params: tf_filter_params) -> int:
+        n = C.c_size_t()
+        _check(lib().tf_workspace_bytes(C.byref(shape), C.byref(params), C.byref(n)), "tf_workspace_bytes")
+        return int(n.value)
+
+    def set_workspace(self, buf: Optional[torch.Tensor]) -> None:
+        self._ws = buf
+        _check(lib().tf_set_workspace(self._h, _ptr(buf), C.c_size_t(0 if buf is None else buf.numel() * buf.element_size())),
+               "tf_set_workspace")
+
+    def ensure_workspace(self, shape: tf_shape, params: tf_filter_params) -> None:
+        need = self.workspace_bytes(shape, params)
+        if self._ws is None or self._ws.numel() < need:
+            self.set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}"))
+
+    # ---- the five entry points -----------------------------------------------------------------
+    def tf_kv_stats(self, shape, params, K, V, sim_k, sim_v, carry: Optional[tf_carry] = None):
+        _check(lib().tf_kv_stats(self._h, C.byref(shape), C.byref(params), _ptr(K), _ptr(V), _ptr(sim_k),
+                                 _ptr(sim_v), None if carry is None else C.byref(carry), _stream()), "tf_kv_stats")
+
+    def tf_score_fuse(self, shape, params, sim_k, sim_v, score):
+        _check(lib().tf_score_fuse(self._h, C.byref(shape), C.byref(params), _ptr(sim_k), _ptr(sim_v),
+                                   _ptr(score), _stream()), "tf_score_fuse")
+
+    def tf_select(self, shape, params, score, keep_mask, kept_idx, n_kept, theta=None):
+        _check(lib().tf_select(self._h, C.byref(shape), C.byref(params), _ptr(score), _ptr(keep_mask),
+                               _ptr(kept_idx), _ptr(n_kept), _ptr(theta), _stream()), "tf_select")
+
+    def tf_pruned_attention(self, shape, params, Q, K, V, kept_idx, n_kept, O):
+        _check(lib().tf_pruned_attention(self._h, C.byref(shape), C.byref(params), _ptr(Q), _ptr(K), _ptr(V),
+                                         _ptr(kept_idx), _ptr(n_kept), _ptr(O), _stream()), "tf_pruned_attention")
+
+    def tf_layer_filter(self, shape, params, Q, K, V, O, score=None, keep_mask=None, kept_idx=None, n_kept=None):
+        _check(lib().tf_layer_filter(self._h, C.byref(shape), C.byref(params), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
+                                     _ptr(score), _ptr(keep_mask), _ptr(kept_idx), _ptr(n_kept), _stream()),
+               "tf_layer_filter")
+
+    def tf_layer_filter_host(self, shape, params, Q, K, V, O, score=None, keep_mask=None, kept_idx=None, n_kept=None):
+        """Host tensors in, host tensors out (copies inside the call; returns after the stream is idle)."""
+        _check(lib().tf_layer_filter_host(self._h, C.byref(shape), C.byref(params), _ptr(Q), _ptr(K), _ptr(V),
+                                          _ptr(O), _ptr(score), _ptr(keep_mask), _ptr(kept_idx), _ptr(n_kept),
+                                          _stream()), "tf_layer_filter_host")
+
+    # ---- status --------------------------------------------------------------------------------
+    def tf_get_status(self, sync: bool = True):
+        det = (C.c_int64 * 4)()
+        code = lib().tf_get_status(self._h, C.c_int(1 if sync else 0), det)
+        return code, dict(code=det[0], where=det[1], nan_count=det[2], launches=det[3])
+
+    def tf_clear_status(self):
+        _check(lib().tf_clear_status(self._h), "tf_clear_status")
+
+    def tf_set_attention_path(self, use_tensor_cores: bool):
+        _check(lib().tf_set_attention_path(self._h, C.c_int(1 if use_tensor_cores else 0)), "tf_set_attention_path")
+
+    @property
+    def launches(self) -> int:
+        return self.tf_get_status(sync=False)[1]["launches"]

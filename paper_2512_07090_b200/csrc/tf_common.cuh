@@ -1,0 +1,122 @@
+// Shared device/host helpers of the Token Filtering CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/tf.h"
+
+namespace tf {
+
+constexpr int kHeadDim = 128;
+constexpr float kNormEps = 1e-8f;   // lower clamp of each norm in the cosine
+
+// Device status record: four 64-bit words {code, where, nan_count, reserved}.
+struct DevStatus {
+    unsigned long long code;
+    unsigned long long where;
+    unsigned long long nan_count;
+    unsigned long long reserved;
+};
+
+__device__ __forceinline__ void report_error(DevStatus* st, int code, unsigned long long where) {
+    if (st == nullptr) return;
+    if (atomicCAS(&st->code, 0ull, (unsigned long long)code) == 0ull) st->where = where;
+}
+
+// ---- element access -------------------------------------------------------------------------
+// Vec16<T>: one 16-byte global load and its expansion to floats (8 bf16 or 4 fp32).
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kPerVec = 4;   // elements per 16-byte vector
+    static constexpr int kVecPerLane = 4;  // 16 dims per lane
+    __device__ static __forceinline__ void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kPerVec = 8;
+    static constexpr int kVecPerLane = 2;
+    // a bf16 is the upper half of the fp32 with the same value
+    __device__ static __forceinline__ void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+        f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+        f[4] = __uint_as_float(r.z << 16); f[5] = __uint_as_float(r.z & 0xffff0000u);
+        f[6] = __uint_as_float(r.w << 16); f[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+
+__device__ __forceinline__ uint4 ldg16(const void* p) {
+    return __ldg(reinterpret_cast<const uint4*>(p));
+}
+// streaming 16-byte load: data that is read exactly once should not displace L1 lines
+__device__ __forceinline__ uint4 ldg16_stream(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// ---- host-side launch bookkeeping --------------------------------------------------------------
+struct Strides3 { long long b, t, h; };
+
+}  // namespace tf
+
+// The opaque context of include/tf.h.
+struct tf_ctx {
+    int device;
+    tf::DevStatus* dev_status;     // device memory, 4 words
+    void* workspace;               // caller-owned (or owned_ws below)
+    size_t workspace_bytes;
+    int use_tensor_cores;          // bf16 attention path
+    long long launches;            // kernels launched through this context
+    // tf_layer_filter_host staging (owned, grown on demand)
+    void* stage;
+    size_t stage_bytes;
+    void* owned_ws;
+    size_t owned_ws_bytes;
+};
+
+// ---- per-kernel launchers (defined in the .cu files, called by tf_api.cu) ----------------------
+namespace tf {
+
+struct ScanPlan {            // how tf_kv_stats tiles a shape
+    int chunk_tokens;        // tokens per CTA tile
+    int n_chains;            // batch * n_kv_heads
+    int n_chunks;            // ceil(seq / chunk_tokens)
+    size_t bytes;            // scratch bytes (ticket + flags + records), 256-aligned
+};
+ScanPlan scan_plan(const tf_shape& s);
+
+cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                            const void* K, const void* V, float* sim_k, float* sim_v,
+                            const tf_carry* carry, void* scan_scratch, cudaStream_t st);
+cudaError_t launch_score_fuse(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                              const float* sim_k, const float* sim_v, float* score, cudaStream_t st);
+cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                          const float* score, uint8_t* keep_mask, int32_t* kept_idx,
+                          int32_t* n_kept, float* theta, cudaStream_t st);
+cudaError_t launch_attention_simt(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                                  const void* Q, const void* K, const void* V,
+                                  const int32_t* kept_idx, const int32_t* n_kept, void* O,
+                                  cudaStream_t st);
+// returns cudaErrorNotSupported when the tensor-core path cannot take this call
+cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                                const void* Q, const void* K, const void* V,
+                                const int32_t* kept_idx, const int32_t* n_kept, void* O,
+                                cudaStream_t st);
+
+}  // namespace tf

@@ -1,0 +1,210 @@
+// Step a4: keep/prune selection and compaction, one CTA per sequence.
+//
+// RATIO mode prunes exactly P = min(E, floor(ratio*S)) eligible tokens: those that come first
+// when eligible tokens are ordered by (score descending, index descending).  The P-th key is
+// found with a 4-pass, 8-bit MSB-first radix select over order-preserving 32-bit keys; tokens
+// whose key equals it are then taken from the highest index down.  THRESHOLD mode prunes the
+// eligible tokens whose score is strictly above threshold[b] (Alg. 1, "skip if s_KV > tau").
+// The retained positions are compacted in ascending order with warp ballots and a block-wide
+// prefix sum.  Scores are re-read from global memory on each pass (they stay in L1/L2).
+#include <math_constants.h>
+
+#include "tf_common.cuh"
+
+namespace tf {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+// Monotone map float -> uint32 (larger score <=> larger key); -0 and +0 share a key.
+__device__ __forceinline__ unsigned int score_key(float s) {
+    if (s == 0.f) s = 0.f;
+    const unsigned int u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_score(unsigned int k) {
+    const unsigned int u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+    return __uint_as_float(u);
+}
+
+struct SelectParams {
+    const float* score;        // [B,S]
+    const uint8_t* eligible;   // [B,S] or null
+    const float* threshold;    // [B] (threshold mode)
+    int S, warmup, mode;
+    long long p_target;        // floor(ratio*S), computed on the host in double
+    uint8_t* keep_mask; int32_t* kept_idx; int32_t* n_kept; float* theta;
+};
+
+// block-wide exclusive prefix over one flag per thread; returns this thread's exclusive rank
+// and the block total (s_warp must hold kSelWarps ints; two barriers inside)
+__device__ __forceinline__ int block_rank(bool flag, int* s_warp, int& total) {
+    const unsigned int bal = __ballot_sync(0xffffffffu, flag);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) s_warp[wid] = __popc(bal);
+    __syncthreads();
+    int before = 0, tot = 0;
+#pragma unroll
+    for (int w2 = 0; w2 < kSelWarps; ++w2) {
+        const int c = s_warp[w2];
+        before += (w2 < wid) ? c : 0;
+        tot += c;
+    }
+    __syncthreads();
+    total = tot;
+    return before + __popc(bal & ((1u << lane) - 1u));
+}
+
+__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectParams p) {
+    __shared__ int hist[256];
+    __shared__ int s_warp[kSelWarps];
+    __shared__ unsigned int s_prefix;
+    __shared__ int s_rank, s_count;
+
+    const int b = blockIdx.x, tid = threadIdx.x, S = p.S;
+    const float* sc = p.score + (size_t)b * S;
+    const uint8_t* el = p.eligible ? p.eligible + (size_t)b * S : nullptr;
+    auto candidate = [&](int t, float s) -> bool {
+        return t >= p.warmup && (el == nullptr || el[t] != 0) && s == s;   // NaN never pruned
+    };
+
+    unsigned int key_thr = 0;   // ratio mode: key of the P-th candidate
+    int take_eq = 0;            // ratio mode: how many tokens with key == key_thr go (highest index first)
+    int n_eq = 0;               // ratio mode: how many candidates have key == key_thr
+    float tau = 0.f;
+    bool nothing = false;       // nothing to prune
+
+    if (p.mode == TF_SELECT_THRESHOLD) {
+        tau = p.threshold[b];
+    } else {
+        // E = number of candidates
+        int e_local = 0;
+        for (int t = tid; t < S; t += kSelThreads) e_local += candidate(t, sc[t]) ? 1 : 0;
+        if (tid == 0) s_count = 0;
+        __syncthreads();
+        e_local = __reduce_add_sync(0xffffffffu, e_local);
+        if ((tid & 31) == 0) atomicAdd(&s_count, e_local);
+        __syncthreads();
+        const long long E = s_count;
+        long long P = p.p_target < E ? p.p_target : E;
+        __syncthreads();
+        if (P <= 0) {
+            nothing = true;
+        } else {
+            // radix select: rank r (1-based from the top) among candidates matching the prefix so far
+            unsigned int prefix = 0, mask = 0;
+            int r = (int)P;
+            for (int shift = 24; shift >= 0; shift -= 8) {
+                for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
+                __syncthreads();
+                for (int t0 = 0; t0 < S; t0 += kSelThreads) {
+                    const int t = t0 + tid;
+                    int bin = 256;   // sentinel: this lane adds nothing
+                    if (t < S) {
+                        const float s = sc[t];
+                        if (candidate(t, s)) {
+                            const unsigned int k = score_key(s);
+                            if ((k & mask) == prefix) bin = (int)((k >> shift) & 255u);
+                        }
+                    }
+                    // scores crowd into a few bins: one shared-memory atomic per distinct bin per warp
+                    const unsigned int same = __match_any_sync(0xffffffffu, bin);
+                    if (bin < 256 && (tid & 31) == __ffs(same) - 1) atomicAdd(&hist[bin], __popc(same));
+                }
+                __syncthreads();
+                // descending inclusive scan of the histogram: the bin where the count reaches r
+                int hval = 0, incl = 0;
+                if (tid < 256) {
+                    hval = hist[255 - tid];
+                    incl = hval;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                        if ((tid & 31) >= o) incl += n;
+                    }
+                    if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
+                }
+                __syncthreads();
+                if (tid < 256) {
+                    int off = 0;
+                    for (int w2 = 0; w2 < (tid >> 5); ++w2) off += s_warp[w2];
+                    incl += off;
+                    const int excl = incl - hval;
+                    if (excl < r && incl >= r) {
+                        s_prefix = prefix | ((unsigned int)(255 - tid) << shift);
+                        s_rank = r - excl;
+                        s_count = hval;
+                    }
+                }
+                __syncthreads();
+                prefix = s_prefix;
+                r = s_rank;
+                n_eq = s_count;
+                mask |= 255u << shift;
+                __syncthreads();
+            }
+            key_thr = prefix;
+            take_eq = r;   // 1 <= r <= n_eq
+        }
+    }
+
+    // ---- sweep in index order: decide, count equals, compact ---------------------------------------
+    int kept_base = 0, eq_base = 0;
+    float th_min = CUDART_INF_F;
+    for (int t0 = 0; t0 < S; t0 += kSelThreads) {
+        const int t = t0 + tid;
+        const bool in = t < S;
+        const float s = in ? sc[t] : 0.f;
+        const bool cand = in && candidate(t, s);
+        bool prune = false;
+        if (p.mode == TF_SELECT_THRESHOLD) {
+            prune = cand && (s > tau);
+        } else if (!nothing) {
+            const unsigned int k = cand ? score_key(s) : 0u;
+            const bool eq = cand && (k == key_thr);
+            int eq_tot;
+            const int eq_rank = block_rank(eq, s_warp, eq_tot) + eq_base;   // 0-based among equals
+            eq_base += eq_tot;
+            // the take_eq equals with the highest index: ranks n_eq-take_eq .. n_eq-1
+            prune = cand && ((k > key_thr) || (eq && eq_rank >= n_eq - take_eq));
+        }
+        if (prune) th_min = fminf(th_min, s);
+        const bool keep = in && !prune;
+        int kept_tot;
+        const int pos = block_rank(keep, s_warp, kept_tot) + kept_base;
+        kept_base += kept_tot;
+        if (in) {
+            p.keep_mask[(size_t)b * S + t] = keep ? 1 : 0;
+            if (keep) p.kept_idx[(size_t)b * S + pos] = t;
+        }
+    }
+    for (int i = kept_base + tid; i < S; i += kSelThreads) p.kept_idx[(size_t)b * S + i] = -1;
+    if (tid == 0) p.n_kept[b] = kept_base;
+    if (p.theta) {
+        // lowest pruned score
+        th_min = -warp_max(-th_min);
+        if ((tid & 31) == 0) s_warp[tid >> 5] = __float_as_int(th_min);
+        __syncthreads();
+        if (tid == 0) {
+            float m = CUDART_INF_F;
+            for (int w2 = 0; w2 < kSelWarps; ++w2) m = fminf(m, __int_as_float(s_warp[w2]));
+            p.theta[b] = m;
+        }
+    }
+}
+
+cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                          const float* score, uint8_t* keep_mask, int32_t* kept_idx,
+                          int32_t* n_kept, float* theta, cudaStream_t st) {
+    if (s.batch == 0) return cudaSuccess;
+    SelectParams sp{};
+    sp.score = score; sp.eligible = p.eligible; sp.threshold = p.threshold;
+    sp.S = s.seq; sp.warmup = p.warmup_tokens; sp.mode = p.select_mode;
+    sp.p_target = (long long)floor(p.prune_ratio * (double)s.seq);
+    sp.keep_mask = keep_mask; sp.kept_idx = kept_idx; sp.n_kept = n_kept; sp.theta = theta;
+    select_kernel<<<s.batch, kSelThreads, 0, st>>>(sp);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace tf

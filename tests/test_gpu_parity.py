@@ -1,0 +1,260 @@
+"""GPU parity: the CUDA path, called through the C-ABI, against the fp64 oracle on the same
+seeded inputs.  Integer results (masks, kept lists, counts) bit-exact; scores within 1e-5;
+attention within 1e-4 (fp32) / 2e-2 (bf16) of the row scale."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_07090_b200 import binding as tfb, workloads as W
+from parity import ATTN_TOL, SCORE_ATOL, Gpu, attn_rel_err, mask_disagreements, oracle_inputs, to_np
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _qkv(B, S, Hq, Hkv, dtype, seed=11, dup=0.25):
+    q, k, v = W.duplicate_qkv(B, S, Hq, Hkv, 128, dup, 0.05, seed=seed, dtype=dtype)
+    return q.to(DEV), k.to(DEV), v.to(DEV)
+
+
+# ------------------------------------------------------------------------------- a1 + a2
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("B,S,Hkv", [(1, 1, 1), (1, 2, 3), (2, 63, 2), (1, 64, 4), (2, 65, 1),
+                                      (3, 333, 5), (2, 1000, 8), (1, 4100, 2)])
+def test_kv_stats_matches_oracle(dtype, B, S, Hkv):
+    q, k, v = _qkv(B, S, Hkv, Hkv, dtype)
+    g = Gpu(q, k, v)
+    g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    g.status_ok()
+    _, kn, vn = oracle_inputs(q, k, v)
+    assert np.abs(to_np(g.sim_k) - oracle.anchor_similarity(kn)).max() < SCORE_ATOL
+    assert np.abs(to_np(g.sim_v) - oracle.anchor_similarity(vn)).max() < SCORE_ATOL
+    g.close()
+
+
+@pytest.mark.parametrize("mode,gamma", [(tfb.TF_ANCHOR_INCL_MEAN, 0.9), (tfb.TF_ANCHOR_EMA, 0.9),
+                                        (tfb.TF_ANCHOR_EMA, 0.8), (tfb.TF_ANCHOR_EMA, 0.95)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_kv_stats_anchor_modes(mode, gamma, dtype):
+    q, k, v = _qkv(2, 517, 4, 4, dtype, seed=5)
+    g = Gpu(q, k, v, anchor_mode=mode, gamma=gamma)
+    g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    g.status_ok()
+    _, kn, vn = oracle_inputs(q, k, v)
+    assert np.abs(to_np(g.sim_k) - oracle.anchor_similarity(kn, mode, gamma)).max() < SCORE_ATOL
+    assert np.abs(to_np(g.sim_v) - oracle.anchor_similarity(vn, mode, gamma)).max() < SCORE_ATOL
+    g.close()
+
+
+def test_kv_stats_head_major_layout_and_carry():
+    """Same values stored [B,H,S,d] (strided view) give the same similarities; two half-sequence
+    calls chained through the carry equal one call; the exported sums are the column sums."""
+    B, S, H = 2, 300, 4
+    q, k, v = _qkv(B, S, H, H, torch.bfloat16, seed=9)
+    kt = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    vt = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert kt.stride() != k.stride()
+    g = Gpu(q, kt, vt)
+    g.ctx.tf_kv_stats(g.shape, g.params, kt, vt, g.sim_k, g.sim_v)
+    _, kn, vn = oracle_inputs(q, k, v)
+    ref_k, sum_k = oracle.anchor_similarity(kn, want_sum_out=True)
+    assert np.abs(to_np(g.sim_k) - ref_k).max() < SCORE_ATOL
+    g.close()
+    # chained halves
+    h = S // 2
+    g1 = Gpu(q[:, :h], k[:, :h], v[:, :h])
+    sk = torch.empty(B, H, 128, device=DEV); sv = torch.empty(B, H, 128, device=DEV)
+    c1 = tfb.tf_carry(None, None, None, sk.data_ptr(), sv.data_ptr())
+    g1.ctx.tf_kv_stats(g1.shape, g1.params, k[:, :h], v[:, :h], g1.sim_k, g1.sim_v, c1)
+    cnt = torch.full((B,), h, dtype=torch.int64, device=DEV)
+    g2 = Gpu(q[:, h:], k[:, h:], v[:, h:])
+    sk2 = torch.empty_like(sk); sv2 = torch.empty_like(sv)
+    c2 = tfb.tf_carry(sk.data_ptr(), sv.data_ptr(), cnt.data_ptr(), sk2.data_ptr(), sv2.data_ptr())
+    g2.ctx.tf_kv_stats(g2.shape, g2.params, k[:, h:], v[:, h:], g2.sim_k, g2.sim_v, c2)
+    g2.status_ok()
+    both = np.concatenate([to_np(g1.sim_k), to_np(g2.sim_k)], 1)
+    assert np.abs(both - ref_k).max() < SCORE_ATOL
+    assert np.abs(to_np(sk2) - sum_k).max() < 1e-3 * max(1.0, np.abs(sum_k).max())
+    g1.close(); g2.close()
+
+
+# ------------------------------------------------------------------------------- a3
+@pytest.mark.parametrize("H", [1, 2, 8, 32, 40])
+@pytest.mark.parametrize("mode", [tfb.TF_FUSE_INVVAR, tfb.TF_FUSE_EQ2_LITERAL, tfb.TF_FUSE_KEY_ONLY,
+                                  tfb.TF_FUSE_VALUE_ONLY, tfb.TF_FUSE_MEAN])
+def test_score_fuse_matches_oracle(H, mode):
+    B, S = 2, 777
+    rng = np.random.default_rng(H * 10 + mode)
+    ck = rng.uniform(-0.3, 0.9, (B, S, H)).astype(np.float32)
+    cv = rng.uniform(-0.3, 0.9, (B, S, H)).astype(np.float32)
+    ck[0, 5] = 0.25; cv[0, 5] = -0.5           # zero variance on both sides
+    q, k, v = _qkv(B, S, H, H, torch.bfloat16)
+    g = Gpu(q, k, v, fuse_mode=mode)
+    g.ctx.tf_score_fuse(g.shape, g.params, torch.from_numpy(ck).to(DEV), torch.from_numpy(cv).to(DEV), g.score)
+    g.status_ok()
+    ref = oracle.score_fuse(ck, cv, mode)
+    assert np.abs(to_np(g.score) - ref).max() < 2e-6
+    g.close()
+
+
+# ------------------------------------------------------------------------------- a4
+def _select_case(score, ratio, warm, elig=None, mode=tfb.TF_SELECT_RATIO, thr=None):
+    """tf_select fed fp32 scores must agree bit for bit with the oracle fed the same values."""
+    B, S = score.shape
+    sc = torch.from_numpy(score).to(DEV)
+    q = torch.zeros(B, S, 1, 128, dtype=torch.bfloat16, device=DEV)
+    kw = dict(prune_ratio=ratio, warmup_tokens=warm, select_mode=mode)
+    el_t = th_t = None
+    if elig is not None:
+        el_t = torch.from_numpy(elig).to(DEV); kw["eligible"] = el_t
+    if thr is not None:
+        th_t = torch.from_numpy(np.asarray(thr, np.float32)).to(DEV); kw["threshold"] = th_t
+    g = Gpu(q, q, q, **kw)
+    g.ctx.tf_select(g.shape, g.params, sc, g.keep, g.idx, g.nk, g.theta)
+    g.status_ok()
+    ref = oracle.select(score.astype(np.float64), ratio, warm, elig, mode, thr)
+    assert np.array_equal(g.keep.cpu().numpy(), ref["keep_mask"])
+    assert np.array_equal(g.idx.cpu().numpy(), ref["kept_idx"])
+    assert np.array_equal(g.nk.cpu().numpy(), ref["n_kept"])
+    assert np.array_equal(g.theta.cpu().numpy().astype(np.float64), ref["theta"])
+    g.close()
+
+
+@pytest.mark.parametrize("S", [1, 2, 31, 1024, 1025, 2048, 5000, 16384])
+@pytest.mark.parametrize("ratio", [0.0, 0.25, 0.5, 0.7, 0.999])
+def test_select_bit_exact_random(S, ratio):
+    rng = np.random.default_rng(S)
+    score = rng.normal(0.2, 0.2, (3, S)).astype(np.float32)
+    _select_case(score, ratio, warm=min(4, S))
+
+
+def test_select_bit_exact_ties_eligibility_nan_threshold():
+    rng = np.random.default_rng(3)
+    S = 3000
+    coarse = np.round(rng.uniform(-1, 1, (2, S)), 1).astype(np.float32)        # many exact ties
+    coarse[0, ::7] = -0.0
+    _select_case(coarse, 0.5, 1)
+    _select_case(np.zeros((2, S), np.float32), 0.3, 2)                          # all equal
+    elig = (rng.uniform(size=(2, S)) < 0.4).astype(np.uint8)
+    _select_case(coarse, 0.7, 10, elig)                                         # capped by eligibility
+    nan = coarse.copy(); nan[1, 100:200] = np.nan
+    _select_case(nan, 0.5, 0)
+    _select_case(coarse, 0.5, 3, None, tfb.TF_SELECT_THRESHOLD, [0.3, -2.0])
+    _select_case(coarse, 0.5, 3, elig, tfb.TF_SELECT_THRESHOLD, [5.0, 0.0])     # nothing / a lot
+
+
+# ------------------------------------------------------------------------------- a5
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5),
+                                                    (1, 257, 8, 2, 0, 0.3), (2, 300, 4, 1, 64, 0.5),
+                                                    (1, 515, 2, 2, 1, 0.7), (1, 200, 4, 2, 0, 0.99)])
+def test_pruned_attention_matches_oracle(dtype, B, S, Hq, Hkv, window, ratio):
+    q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=S)
+    qn, kn, vn = oracle_inputs(q, k, v)
+    ref = oracle.layer_filter(qn, kn, vn, prune_ratio=ratio, warmup_tokens=1, window=window)
+    g = Gpu(q, k, v, window=window)
+    idx = torch.from_numpy(ref["kept_idx"]).to(DEV)
+    nk = torch.from_numpy(ref["n_kept"]).to(DEV)
+    g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
+    g.status_ok()
+    o = to_np(g.O)
+    assert np.isfinite(o).all()
+    assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
+    assert np.all(o[ref["keep_mask"] == 0] == 0.0)
+    g.close()
+
+
+def test_pruned_attention_nothing_kept_and_everything_kept():
+    q, k, v = _qkv(2, 70, 2, 2, torch.bfloat16)
+    g = Gpu(q, k, v)
+    idx = torch.full((2, 70), -1, dtype=torch.int32, device=DEV)
+    idx[1] = torch.arange(70, dtype=torch.int32, device=DEV)
+    nk = torch.tensor([0, 70], dtype=torch.int32, device=DEV)
+    g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
+    o = to_np(g.O)
+    assert np.all(o[0] == 0)
+    qn, kn, vn = oracle_inputs(q, k, v)
+    dense = oracle.pruned_attention(qn, kn, vn, np.ones((2, 70), np.uint8))
+    assert attn_rel_err(o[1], dense[1]) < ATTN_TOL[torch.bfloat16]
+    g.close()
+
+
+# ------------------------------------------------------------------------------- whole layer
+def _layer_case(q, k, v, window=0, **kw):
+    qn, kn, vn = oracle_inputs(q, k, v)
+    okw = {a: b for a, b in kw.items()}
+    ref = oracle.layer_filter(qn, kn, vn, window=window, **okw)
+    g = Gpu(q, k, v, window=window, **kw)
+    g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
+    g.status_ok()
+    assert np.abs(to_np(g.score) - ref["score"]).max() < SCORE_ATOL
+    n_mis, n_out = mask_disagreements(g.keep.cpu().numpy(), ref)
+    assert n_out == 0, f"{n_mis} keep/prune disagreements, {n_out} outside the 1e-6 band around theta"
+    keep = g.keep.cpu().numpy()
+    idx = g.idx.cpu().numpy(); nk = g.nk.cpu().numpy()
+    for b in range(keep.shape[0]):
+        assert np.array_equal(idx[b, :nk[b]], np.nonzero(keep[b])[0]) and np.all(idx[b, nk[b]:] == -1)
+    if n_mis == 0:
+        assert attn_rel_err(to_np(g.O), ref["O"]) < ATTN_TOL[q.dtype]
+    else:   # compare attention on the oracle's own kept set
+        g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, torch.from_numpy(ref["kept_idx"]).to(DEV),
+                                  torch.from_numpy(ref["n_kept"]).to(DEV), g.O)
+        assert attn_rel_err(to_np(g.O), ref["O"]) < ATTN_TOL[q.dtype]
+    g.close()
+    return n_mis
+
+
+def test_layer_filter_config1_fp32():
+    """Config 1 in full: B1 S128 32 heads fp32, 25% near-duplicates, 50% pruning."""
+    wl = W.WORKLOADS["c1"]
+    _, q, k, v = next(wl.layer_qkv([0], DEV))
+    _layer_case(q, k, v, prune_ratio=0.5, warmup_tokens=4)
+    _layer_case(q, k, v, prune_ratio=0.5, warmup_tokens=4, fuse_mode=tfb.TF_FUSE_EQ2_LITERAL)
+
+
+@pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 777, 8, 8, 0, 0.5), (2, 1111, 8, 2, 0, 0.3),
+                                                    (2, 900, 8, 2, 0, 0.7), (2, 1500, 8, 2, 256, 0.5),
+                                                    (1, 640, 10, 10, 0, 0.25), (1, 333, 4, 4, 0, 0.0)])
+def test_layer_filter_reduced_shapes_bf16(B, S, Hq, Hkv, window, ratio):
+    q, k, v = _qkv(B, S, Hq, Hkv, torch.bfloat16, seed=S + Hq)
+    _layer_case(q, k, v, window=window, prune_ratio=ratio, warmup_tokens=4)
+
+
+def test_layer_filter_host_entry_matches_device_entry():
+    q, k, v = W.duplicate_qkv(2, 400, 8, 2, 128, 0.25, 0.05, seed=21, dtype=torch.bfloat16)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    g = Gpu(qd, kd, vd, prune_ratio=0.5, warmup_tokens=4)
+    g.ctx.tf_layer_filter(g.shape, g.params, qd, kd, vd, g.O, g.score, g.keep, g.idx, g.nk)
+    torch.cuda.synchronize()
+    qh, kh, vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+    oh = torch.empty_like(qh).pin_memory()
+    sh = torch.empty(2, 400).pin_memory(); mh = torch.empty(2, 400, dtype=torch.uint8).pin_memory()
+    ih = torch.empty(2, 400, dtype=torch.int32).pin_memory(); nh = torch.empty(2, dtype=torch.int32).pin_memory()
+    hs = tfb.make_shape(qh, kh, vh, oh)
+    g.ctx.tf_layer_filter_host(hs, g.params, qh, kh, vh, oh, sh, mh, ih, nh)
+    assert torch.equal(oh, g.O.cpu()) and torch.equal(sh, g.score.cpu()) and torch.equal(mh, g.keep.cpu())
+    assert torch.equal(ih, g.idx.cpu()) and torch.equal(nh, g.nk.cpu())
+    g.close()
+
+
+def test_device_rejects_bad_arguments_without_launching():
+    q, k, v = _qkv(1, 64, 2, 2, torch.bfloat16)
+    g = Gpu(q, k, v)
+    L = tfb.lib()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    n0 = g.ctx.launches
+    bad = tfb.default_params(prune_ratio=1.0)
+    assert L.tf_layer_filter(g.ctx._h, C.byref(g.shape), C.byref(bad), *[C.c_void_p(t.data_ptr()) for t in (q, k, v, g.O)],
+                             None, None, None, None, st) == tfb.TF_ERR_INVALID_ARG
+    assert L.tf_kv_stats(g.ctx._h, C.byref(g.shape), C.byref(g.params), C.c_void_p(k.data_ptr() + 2),
+                         C.c_void_p(v.data_ptr()), C.c_void_p(g.sim_k.data_ptr()), C.c_void_p(g.sim_v.data_ptr()),
+                         None, st) == tfb.TF_ERR_UNSUPPORTED
+    g.ctx.set_workspace(None)
+    assert L.tf_kv_stats(g.ctx._h, C.byref(g.shape), C.byref(g.params), C.c_void_p(k.data_ptr()),
+                         C.c_void_p(v.data_ptr()), C.c_void_p(g.sim_k.data_ptr()), C.c_void_p(g.sim_v.data_ptr()),
+                         None, st) == tfb.TF_ERR_WORKSPACE
+    assert g.ctx.launches == n0
+    g.close()
