@@ -28,8 +28,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-DTF_BUILD",
-           "-o", LIB] + sources() + ["-lcuda"]
+           "-shared", "-Xcompiler", "-fPIC", "-DTF_BUILD", "-o", LIB] + sources()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -119,9 +119,8 @@ tf_status tf_create(tf_ctx** out, int device) {
     if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return TF_ERR_CUDA;
     DeviceGuard g(device);
     if (!g.ok) return TF_ERR_CUDA;
-    tf_ctx* c = new (std::nothrow) tf_ctx();
+    tf_ctx* c = new (std::nothrow) tf_ctx{};
     if (!c) return TF_ERR_CUDA;
-    memset(c, 0, sizeof(*c));
     c->device = device;
     c->use_tensor_cores = 1;
     if (cudaMalloc(reinterpret_cast<void**>(&c->dev_status), sizeof(DevStatus)) != cudaSuccess ||
@@ -157,6 +156,8 @@ tf_status tf_set_workspace(tf_ctx* ctx, void* device_ptr, size_t bytes) {
     if (device_ptr && (reinterpret_cast<uintptr_t>(device_ptr) & 255u)) return TF_ERR_INVALID_ARG;
     ctx->workspace = device_ptr;
     ctx->workspace_bytes = device_ptr ? bytes : 0;
+    ctx->scan_user = tf::ScanScratch();
+    ctx->scan_user.ptr = device_ptr;
     return TF_OK;
 }
 
@@ -172,7 +173,7 @@ tf_status tf_kv_stats(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params
     if (!ctx->workspace || ctx->workspace_bytes < scan_plan(*shape).bytes) return TF_ERR_WORKSPACE;
     DeviceGuard g(ctx->device);
     if (!g.ok) return TF_ERR_CUDA;
-    cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, carry, ctx->workspace,
+    cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, carry, &ctx->scan_user,
                                     static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
 }
@@ -248,7 +249,8 @@ tf_status tf_layer_filter(tf_ctx* ctx, const tf_shape* shape, const tf_filter_pa
     if (!n_kept) n_kept = reinterpret_cast<int32_t*>(ws + w.n_kept);
     float* theta = reinterpret_cast<float*>(ws + w.theta);
 
-    cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, nullptr, ws + w.scan, st);
+    ScanScratch* scan = (ctx->workspace == ctx->owned_ws && ctx->owned_ws) ? &ctx->scan_owned : &ctx->scan_user;
+    cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, nullptr, scan, st);
     if (e == cudaSuccess) e = launch_score_fuse(ctx, *shape, *params, sim_k, sim_v, score, st);
     if (e == cudaSuccess) e = launch_select(ctx, *shape, *params, score, keep_mask, kept_idx, n_kept, theta, st);
     if (e != cudaSuccess) return TF_ERR_CUDA;
@@ -291,6 +293,8 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         if (ctx->owned_ws) { cudaStreamSynchronize(st); cudaFree(ctx->owned_ws); ctx->owned_ws = nullptr; ctx->owned_ws_bytes = 0; }
         if (cudaMalloc(&ctx->owned_ws, w.total) != cudaSuccess) return TF_ERR_CUDA;
         ctx->owned_ws_bytes = w.total;
+        ctx->scan_owned = tf::ScanScratch();
+        ctx->scan_owned.ptr = ctx->owned_ws;
     }
     char* base = static_cast<char*>(ctx->stage);
     void* dQ = base; void* dO = base + qb; void* dK = base + 2 * qb; void* dV = base + 2 * qb + kb;

@@ -75,12 +75,25 @@ struct Strides3 { long long b, t, h; };
 
 }  // namespace tf
 
+namespace tf {
+// Host-side bookkeeping of one scan scratch region (the first section of a workspace).
+struct ScanScratch {
+    void* ptr = nullptr;
+    size_t bytes = 0;               // bytes of the region the scan may use (cleared on first use)
+    unsigned int epoch = 0;         // tag of the latest launch
+    unsigned int ticket_base = 0;   // value of the ticket word before the next launch
+    bool needs_clear = true;
+};
+}  // namespace tf
+
 // The opaque context of include/tf.h.
 struct tf_ctx {
     int device;
     tf::DevStatus* dev_status;     // device memory, 4 words
-    void* workspace;               // caller-owned (or owned_ws below)
+    void* workspace;               // caller-owned
     size_t workspace_bytes;
+    tf::ScanScratch scan_user;     // scan bookkeeping of the caller's workspace
+    tf::ScanScratch scan_owned;    // ... and of owned_ws
     int use_tensor_cores;          // bf16 attention path
     long long launches;            // kernels launched through this context
     // tf_layer_filter_host staging (owned, grown on demand)
@@ -97,13 +110,14 @@ struct ScanPlan {            // how tf_kv_stats tiles a shape
     int chunk_tokens;        // tokens per CTA tile
     int n_chains;            // batch * n_kv_heads
     int n_chunks;            // ceil(seq / chunk_tokens)
-    size_t bytes;            // scratch bytes (ticket + flags + records), 256-aligned
+    size_t agg_offset, prefix_offset;   // byte offsets of the record arrays in the scratch
+    size_t bytes;            // scratch bytes (ticket word + records), 256-aligned
 };
 ScanPlan scan_plan(const tf_shape& s);
 
 cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                             const void* K, const void* V, float* sim_k, float* sim_v,
-                            const tf_carry* carry, void* scan_scratch, cudaStream_t st);
+                            const tf_carry* carry, ScanScratch* scan_scratch, cudaStream_t st);
 cudaError_t launch_score_fuse(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                               const float* sim_k, const float* sim_v, float* score, cudaStream_t st);
 cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,

@@ -3,16 +3,22 @@
 // kv_stats_kernel: single pass over K and V.  The running sum of past tokens (the anchor up to
 // a scale factor, Alg. 1 "AnchorK <- mean(K)") is a prefix sum along the sequence per (batch,
 // kv head, dim).  A CTA owns one chunk of tokens of one head, keeps that chunk in registers,
-// and resolves the sum of everything before its chunk with a chained scan: it publishes its
-// chunk aggregate, then looks back over its predecessors' records until it meets one whose
-// inclusive prefix is known.  Tiles are handed out by an atomic ticket, chunk index slowest,
-// so every predecessor of a running tile has itself started: the look-back cannot deadlock,
+// and resolves the sum of everything before its chunk with a chained scan over per-chunk
+// records in global memory:
+//   - every chunk publishes its aggregate; every kAnchorEvery-th chunk also publishes its
+//     exclusive prefix P;
+//   - chunk c takes P of the nearest earlier anchor chunk a and adds the aggregates a..c-1 in
+//     ascending order.  The association is fixed, so results do not depend on timing.
+// A record is 128 16-byte packets {k value, v value, tag, 0}; a packet is valid when its tag is
+// this launch's epoch, so value and validity arrive in one load and nothing is cleared between
+// launches.  Tiles are handed out by an atomic ticket, chunk index slowest, so every record a
+// running tile waits for belongs to a tile that has itself started: the waits cannot deadlock,
 // and every wait is bounded anyway (on expiry the kernel records TF_ERR_TIMEOUT and goes on).
 //
 // Inside the CTA, 8 lanes share a token row (16 dims each, two 16-byte loads for bf16) and 16
 // such groups take consecutive runs of tokens; the groups' local sums are scanned through
 // shared memory.  Bytes moved: K and V once, 8 bytes of similarity per (token, head) out,
-// about 1-2 KiB of scan records per 32 KiB tile.
+// 2 KiB of record per 32 KiB tile.
 #include "tf_common.cuh"
 
 namespace tf {
@@ -26,7 +32,8 @@ template <typename T> struct ScanCfg;
 template <> struct ScanCfg<float> { static constexpr int kTokPerGroup = 2; };
 template <> struct ScanCfg<__nv_bfloat16> { static constexpr int kTokPerGroup = 4; };
 
-enum : int { kFlagNone = 0, kFlagAggregate = 1, kFlagPrefix = 2, kFlagTimeout = -1 };
+constexpr int kAnchorEvery = 8;   // every 8th chunk of a chain publishes its exclusive prefix
+constexpr int kPollBatch = 4;     // record packets requested together while looking back
 
 struct ScanParams {
     const void* K; const void* V;
@@ -37,18 +44,39 @@ struct ScanParams {
     const float* sum_k_in; const float* sum_v_in; const long long* count_in;
     float* sum_k_out; float* sum_v_out;
     float* sim_k; float* sim_v;
-    unsigned int* ticket; int* flags; float* records;   // records[tile][agg|prefix][k|v][128]
+    unsigned int* ticket; unsigned int ticket_base, epoch;
+    uint4* agg_rec;      // [tile][128] packets, tile = chunk * n_chains + chain
+    uint4* prefix_rec;   // [(chunk / kAnchorEvery) * n_chains + chain][128] packets
     DevStatus* status;
     int max_polls;
 };
 
-__device__ __forceinline__ int ld_acquire(const int* p) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
+// 16-byte packets go straight to / come straight from L2 as single transactions
+__device__ __forceinline__ uint4 ld_packet(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
+    return r;
 }
-__device__ __forceinline__ void st_release(int* p, int v) {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_packet(uint4* p, float k, float v, unsigned int tag) {
+    asm volatile("st.volatile.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(__float_as_uint(k)), "r"(__float_as_uint(v)), "r"(tag), "r"(0u) : "memory");
+}
+// wait (bounded) until the packet at p carries this launch's tag
+__device__ __forceinline__ uint4 wait_packet(const uint4* p, uint4 first, unsigned int epoch, int max_polls,
+                                             DevStatus* status, unsigned long long where) {
+    uint4 r = first;
+    int polls = 0;
+    while (r.z != epoch) {
+        if (++polls > max_polls) {
+            report_error(status, TF_ERR_TIMEOUT, where);
+            r = make_uint4(0u, 0u, epoch, 0u);
+            break;
+        }
+        __nanosleep(32);
+        r = ld_packet(p);
+    }
+    return r;
 }
 
 // dim owned by (vector j, lane l, element e): vectors of one row are interleaved across the
@@ -65,10 +93,9 @@ __global__ void __launch_bounds__(kScanThreads, 4) kv_stats_kernel(const ScanPar
 
     __shared__ __align__(16) float sub[2][kGroups][kHeadDim];
     __shared__ unsigned int s_ticket;
-    __shared__ int s_flag;
 
     const int tid = threadIdx.x, g = tid >> 3, l = tid & 7;
-    if (tid == 0) s_ticket = atomicAdd(p.ticket, 1u);
+    if (tid == 0) s_ticket = atomicAdd(p.ticket, 1u) - p.ticket_base;
     __syncthreads();
     const unsigned int tile = s_ticket;
     const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
@@ -144,72 +171,45 @@ __global__ void __launch_bounds__(kScanThreads, 4) kv_stats_kernel(const ScanPar
         a_chunk *= f;
     }
 
-    float* rec = p.records + (size_t)tile * (4 * kHeadDim);   // [agg k, agg v, prefix k, prefix v]
+    // every chunk but the last of its chain publishes its aggregate
+    if (c + 1 < p.n_chunks) st_packet(p.agg_rec + (size_t)tile * kHeadDim + tid, agg_k, agg_v, p.epoch);
+
     float carry_k = 0.f, carry_v = 0.f;
     if (c == 0) {
         if (p.sum_k_in) carry_k = p.sum_k_in[(size_t)chain * kHeadDim + tid];
         if (p.sum_v_in) carry_v = p.sum_v_in[(size_t)chain * kHeadDim + tid];
     } else {
-        long long pred = (long long)tile - p.n_chains;
-        // a full predecessor chunk decays the carry by decay^CH
-        float a_full = 1.f;
+        const int a0 = ((c - 1) / kAnchorEvery) * kAnchorEvery;   // nearest earlier anchor chunk
+        float a_full = 1.f;                                        // decay of one full chunk
         if (EMA) { for (int n = 0; n < CH; ++n) a_full *= a; }
-        float fac = 1.f;
-        bool published = false;
-        for (;;) {
-            if (tid == 0) {
-                int f = ld_acquire(p.flags + pred);
-                if (f == kFlagNone && published) {
-                    int polls = 0;
-                    while ((f = ld_acquire(p.flags + pred)) == kFlagNone) {
-                        if (++polls > p.max_polls) { f = kFlagTimeout; break; }
-                        __nanosleep(64);
-                    }
+        const uint4* prec = p.prefix_rec + ((size_t)(a0 / kAnchorEvery) * p.n_chains + chain) * kHeadDim + tid;
+        uint4 pfirst = ld_packet(prec);
+        float Ak = 0.f, Av = 0.f, decay_to_here = 1.f;
+        for (int j0 = a0; j0 < c; j0 += kPollBatch) {
+            uint4 r[kPollBatch];
+#pragma unroll
+            for (int u = 0; u < kPollBatch; ++u)
+                if (j0 + u < c) r[u] = ld_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
+#pragma unroll
+            for (int u = 0; u < kPollBatch; ++u) {
+                if (j0 + u < c) {
+                    r[u] = wait_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u],
+                                       p.epoch, p.max_polls, p.status, tile);
+                    Ak = EMA ? fmaf(a_full, Ak, __uint_as_float(r[u].x)) : Ak + __uint_as_float(r[u].x);
+                    Av = EMA ? fmaf(a_full, Av, __uint_as_float(r[u].y)) : Av + __uint_as_float(r[u].y);
+                    decay_to_here *= a_full;
                 }
-                s_flag = f;
             }
-            __syncthreads();
-            const int f = s_flag;
-            __syncthreads();
-            if (f == kFlagNone) {
-                // predecessor not ready yet: let our successors see our aggregate, then wait
-                __stcg(rec + tid, agg_k);
-                __stcg(rec + kHeadDim + tid, agg_v);
-                __threadfence();
-                __syncthreads();
-                if (tid == 0) st_release(p.flags + tile, kFlagAggregate);
-                published = true;
-                continue;
-            }
-            if (f == kFlagTimeout) {
-                if (tid == 0) report_error(p.status, TF_ERR_TIMEOUT, tile);
-                break;
-            }
-            const float* prec = p.records + (size_t)pred * (4 * kHeadDim);
-            if (f == kFlagPrefix) {
-                carry_k = fmaf(fac, __ldcg(prec + 2 * kHeadDim + tid), carry_k);
-                carry_v = fmaf(fac, __ldcg(prec + 3 * kHeadDim + tid), carry_v);
-                break;
-            }
-            carry_k = fmaf(fac, __ldcg(prec + tid), carry_k);
-            carry_v = fmaf(fac, __ldcg(prec + kHeadDim + tid), carry_v);
-            fac *= a_full;
-            pred -= p.n_chains;
-            if (pred < 0) break;   // cannot happen: chunk 0 only ever publishes a prefix
         }
+        pfirst = wait_packet(prec, pfirst, p.epoch, p.max_polls, p.status, tile);
+        carry_k = EMA ? fmaf(decay_to_here, __uint_as_float(pfirst.x), Ak) : __uint_as_float(pfirst.x) + Ak;
+        carry_v = EMA ? fmaf(decay_to_here, __uint_as_float(pfirst.y), Av) : __uint_as_float(pfirst.y) + Av;
     }
-    {
-        const float incl_k = fmaf(a_chunk, carry_k, agg_k), incl_v = fmaf(a_chunk, carry_v, agg_v);
-        if (c + 1 < p.n_chunks) {
-            __stcg(rec + 2 * kHeadDim + tid, incl_k);
-            __stcg(rec + 3 * kHeadDim + tid, incl_v);
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) st_release(p.flags + tile, kFlagPrefix);
-        } else {
-            if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = incl_k;
-            if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = incl_v;
-        }
+    if (c % kAnchorEvery == 0 && c + 1 < p.n_chunks)
+        st_packet(p.prefix_rec + ((size_t)(c / kAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, p.epoch);
+    if (c + 1 == p.n_chunks) {
+        if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = fmaf(a_chunk, carry_k, agg_k);
+        if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = fmaf(a_chunk, carry_v, agg_v);
     }
     // exclusive scan of the groups' contributions, seeded with the carry
     {
@@ -291,21 +291,34 @@ ScanPlan scan_plan(const tf_shape& s) {
     pl.n_chains = s.batch * s.n_kv_heads;
     pl.n_chunks = (s.seq + pl.chunk_tokens - 1) / pl.chunk_tokens;
     const size_t tiles = (size_t)pl.n_chains * (size_t)pl.n_chunks;
-    size_t flags = 256 + ((tiles * sizeof(int) + 255) / 256) * 256;   // ticket word + flags
-    pl.bytes = flags + tiles * 4 * kHeadDim * sizeof(float);
+    const size_t anchors = (size_t)pl.n_chains * (size_t)((pl.n_chunks + kAnchorEvery - 1) / kAnchorEvery);
+    pl.agg_offset = 256;                                                  // after the ticket word
+    pl.prefix_offset = pl.agg_offset + tiles * kHeadDim * sizeof(uint4);
+    pl.bytes = pl.prefix_offset + anchors * kHeadDim * sizeof(uint4);
     pl.bytes = (pl.bytes + 255) / 256 * 256;
     return pl;
 }
 
 cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                             const void* K, const void* V, float* sim_k, float* sim_v,
-                            const tf_carry* carry, void* scan_scratch, cudaStream_t st) {
+                            const tf_carry* carry, ScanScratch* ws, cudaStream_t st) {
     const ScanPlan pl = scan_plan(s);
     const size_t tiles = (size_t)pl.n_chains * (size_t)pl.n_chunks;
     if (tiles == 0) return cudaSuccess;
-    const size_t flag_bytes = 256 + ((tiles * sizeof(int) + 255) / 256) * 256;
-    cudaError_t e = cudaMemsetAsync(scan_scratch, 0, flag_bytes, st);
-    if (e != cudaSuccess) return e;
+    if (tiles > 0x7fffffffu) return cudaErrorInvalidValue;
+    // Tags make stale records harmless, except in memory this library has never written: clear a
+    // scratch region once when it is first used (and whenever the 32-bit epoch wraps).
+    // The region is also cleared when its extent changes: another shape's layout may have put
+    // other data where this shape keeps records.
+    if (ws->needs_clear || ws->bytes != pl.bytes || ws->epoch == 0xffffffffu) {
+        cudaError_t e = cudaMemsetAsync(ws->ptr, 0, pl.bytes, st);
+        if (e != cudaSuccess) return e;
+        ws->needs_clear = false;
+        ws->bytes = pl.bytes;
+        ws->epoch = 0;
+        ws->ticket_base = 0;
+    }
+    ws->epoch += 1;
 
     ScanParams sp{};
     sp.K = K; sp.V = V;
@@ -322,11 +335,15 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
         sp.sum_k_out = carry->sum_k_out; sp.sum_v_out = carry->sum_v_out;
     }
     sp.sim_k = sim_k; sp.sim_v = sim_v;
-    sp.ticket = reinterpret_cast<unsigned int*>(scan_scratch);
-    sp.flags = reinterpret_cast<int*>(reinterpret_cast<char*>(scan_scratch) + 256);
-    sp.records = reinterpret_cast<float*>(reinterpret_cast<char*>(scan_scratch) + flag_bytes);
+    char* base = static_cast<char*>(ws->ptr);
+    sp.ticket = reinterpret_cast<unsigned int*>(base);
+    sp.ticket_base = ws->ticket_base;
+    sp.epoch = ws->epoch;
+    sp.agg_rec = reinterpret_cast<uint4*>(base + pl.agg_offset);
+    sp.prefix_rec = reinterpret_cast<uint4*>(base + pl.prefix_offset);
     sp.status = ctx->dev_status;
-    sp.max_polls = 1 << 20;   // ~64 ns apart plus an L2 round trip each: of the order of a second
+    sp.max_polls = 1 << 20;   // >= 32 ns apart plus an L2 round trip each: of the order of a second
+    ws->ticket_base += (unsigned int)tiles;   // the ticket word only ever counts up (mod 2^32)
 
     const dim3 grid((unsigned)tiles), block(kScanThreads);
     if (s.dtype == TF_BF16) {

@@ -115,7 +115,8 @@ def _select_case(score, ratio, warm, elig=None, mode=tfb.TF_SELECT_RATIO, thr=No
     g = Gpu(q, q, q, **kw)
     g.ctx.tf_select(g.shape, g.params, sc, g.keep, g.idx, g.nk, g.theta)
     g.status_ok()
-    ref = oracle.select(score.astype(np.float64), ratio, warm, elig, mode, thr)
+    thr64 = None if thr is None else np.asarray(thr, np.float32).astype(np.float64)   # the same fp32 values
+    ref = oracle.select(score.astype(np.float64), ratio, warm, elig, mode, thr64)
     assert np.array_equal(g.keep.cpu().numpy(), ref["keep_mask"])
     assert np.array_equal(g.idx.cpu().numpy(), ref["kept_idx"])
     assert np.array_equal(g.nk.cpu().numpy(), ref["n_kept"])
@@ -131,31 +132,40 @@ def test_select_bit_exact_random(S, ratio):
     _select_case(score, ratio, warm=min(4, S))
 
 
-def test_select_bit_exact_ties_eligibility_nan_threshold():
+@pytest.mark.parametrize("case", ["ties", "all_equal", "eligible", "nan", "threshold", "threshold_eligible"])
+def test_select_bit_exact_ties_eligibility_nan_threshold(case):
     rng = np.random.default_rng(3)
     S = 3000
     coarse = np.round(rng.uniform(-1, 1, (2, S)), 1).astype(np.float32)        # many exact ties
     coarse[0, ::7] = -0.0
-    _select_case(coarse, 0.5, 1)
-    _select_case(np.zeros((2, S), np.float32), 0.3, 2)                          # all equal
     elig = (rng.uniform(size=(2, S)) < 0.4).astype(np.uint8)
-    _select_case(coarse, 0.7, 10, elig)                                         # capped by eligibility
-    nan = coarse.copy(); nan[1, 100:200] = np.nan
-    _select_case(nan, 0.5, 0)
-    _select_case(coarse, 0.5, 3, None, tfb.TF_SELECT_THRESHOLD, [0.3, -2.0])
-    _select_case(coarse, 0.5, 3, elig, tfb.TF_SELECT_THRESHOLD, [5.0, 0.0])     # nothing / a lot
+    if case == "ties":
+        _select_case(coarse, 0.5, 1)
+    elif case == "all_equal":
+        _select_case(np.zeros((2, S), np.float32), 0.3, 2)
+    elif case == "eligible":
+        _select_case(coarse, 0.7, 10, elig)                                     # capped by eligibility
+    elif case == "nan":
+        nan = coarse.copy(); nan[1, 100:200] = np.nan
+        _select_case(nan, 0.5, 0)
+    elif case == "threshold":
+        _select_case(coarse, 0.5, 3, None, tfb.TF_SELECT_THRESHOLD, [0.3, -2.0])
+    else:
+        _select_case(coarse, 0.5, 3, elig, tfb.TF_SELECT_THRESHOLD, [5.0, 0.0])  # nothing / a lot
 
 
 # ------------------------------------------------------------------------------- a5
-@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, True), (torch.bfloat16, False), (torch.float32, False)])
 @pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5),
                                                     (1, 257, 8, 2, 0, 0.3), (2, 300, 4, 1, 64, 0.5),
-                                                    (1, 515, 2, 2, 1, 0.7), (1, 200, 4, 2, 0, 0.99)])
-def test_pruned_attention_matches_oracle(dtype, B, S, Hq, Hkv, window, ratio):
+                                                    (1, 515, 2, 2, 1, 0.7), (1, 200, 4, 2, 0, 0.99),
+                                                    (1, 1300, 4, 2, 300, 0.5), (2, 1024, 2, 1, 0, 0.25)])
+def test_pruned_attention_matches_oracle(dtype, tensor_cores, B, S, Hq, Hkv, window, ratio):
     q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=S)
     qn, kn, vn = oracle_inputs(q, k, v)
     ref = oracle.layer_filter(qn, kn, vn, prune_ratio=ratio, warmup_tokens=1, window=window)
     g = Gpu(q, k, v, window=window)
+    g.ctx.tf_set_attention_path(tensor_cores)
     idx = torch.from_numpy(ref["kept_idx"]).to(DEV)
     nk = torch.from_numpy(ref["n_kept"]).to(DEV)
     g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
