@@ -1,22 +1,31 @@
 // Step a5 on the 5th-generation tensor cores: bf16 causal (optionally windowed) attention for
 // retained tokens only, head_dim 128.
 //
-// One CTA owns 128 consecutive entries of a sequence's retained list for one query head.  The
-// query rows are gathered (they are scattered in the sequence) into shared memory in the
-// 128-byte-swizzled K-major operand layout; K and V tiles of 128 keys are fetched by TMA through
-// tensor maps over the caller's strided K/V and consumed in place by tcgen05.mma:
-//     S = Q K^T   (A = Q, B = K, both K-major)          -> TMEM, two buffers
-//     O += P V    (A = P from shared memory, B = V MN-major, i.e. as it lies in memory) -> TMEM
-// Thread r owns row r: it reads its S row from TMEM, applies the row's own causal / window
-// limits (row r attends keys up to ITS token position, not the tile diagonal), runs the online
-// softmax in fp32, rescales its O row in TMEM when the running maximum moved, and writes P as
-// bf16.  QK^T of the next tile is issued before the softmax of the current one, so tensor work
-// overlaps the exponentials.  The epilogue normalises, converts to bf16 and scatters rows back
-// to their token positions; rows of pruned tokens between two retained tokens are zeroed by the
-// thread that owns the later one (Section 3.2: skipped tokens' attention output is zero).
+// One CTA owns 256 consecutive entries of a sequence's retained list for one query head, as two
+// 128-row Q tiles that share every K/V tile.  Warp roles:
+//   warps 0-3 / 4-7  softmax group of Q tile 0 / 1 (thread r owns row r of its tile)
+//   warp 8           issues every tcgen05.mma (one lane)
+//   warp 9           TMA producer: K and V tiles of 128 keys into a 4-slot ring (one lane)
+//   warps 10-11      idle; they complete the warpgroup whose registers go to the softmax groups
+// The query rows are gathered (they are scattered in the sequence) into shared memory in the
+// 128-byte-swizzled K-major operand layout.  Per K/V tile j and Q tile i:
+//     S_i = Q_i K_j^T      A, B from shared memory (K-major)            -> TMEM, 128 columns
+//     O_i += P_i V_j       A = P_i from TMEM (bf16, written over S_i),  B = V as it lies in
+//                          memory (MN-major)                            -> TMEM, 128 columns
+// issued in the order PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1): the tensor pipe works on one Q tile
+// while the other tile's softmax group runs its exponentials.  The pipe executes in issue order,
+// so S_i(j+1) is never produced before PV_i(j) has consumed P_i(j), and once a softmax group sees
+// S_i(j) it may rescale O_i (PV_i(j-1) is complete).
+// Softmax (fp32): row r applies ITS OWN causal / window limits (a tile of retained rows spans
+// about 128/(1-ratio) positions), keeps a running reference maximum that is only moved (and O_i
+// only rescaled) when the tile maximum exceeds it by more than 2^8, and writes P as bf16 pairs
+// straight back into TMEM.  A Q tile skips K/V tiles none of its rows can see.  The epilogue
+// normalises, converts to bf16 and scatters rows to their token positions; rows of pruned tokens
+// between two retained tokens are zeroed by the thread that owns the later one (Section 3.2:
+// a skipped token's attention output is zero).
 //
 // Every mbarrier wait is bounded by a cycle budget; on expiry the CTA records TF_ERR_TIMEOUT,
-// stops waiting, releases its TMEM and exits.
+// stops waiting, lets copies in flight land, releases its TMEM and exits.
 #include <cuda.h>
 
 #include "tf_common.cuh"
@@ -24,13 +33,18 @@
 namespace tf {
 namespace {
 
-constexpr int kTileM = 128;           // query rows per CTA
-constexpr int kTileN = 128;           // keys per tile
+constexpr int kTileM = 128;           // rows per Q tile
+constexpr int kQTiles = 2;            // Q tiles per CTA
+constexpr int kTileN = 128;           // keys per K/V tile
 constexpr int kHalfBytes = 128 * 128; // one [128 rows][128 B] swizzled block (64 bf16 per row)
 constexpr int kTileBytes = 2 * kHalfBytes;
-constexpr int kKvStages = 2;
-constexpr uint32_t kTmemCols = 512;
+constexpr int kStages = 4;            // ring slots, used K(j), V(j), K(j+1), V(j+1), ...
+constexpr int kSoftmaxThreads = kQTiles * kTileM;
+constexpr int kThreads = kSoftmaxThreads + 128;   // third warpgroup: MMA warp, TMA warp, two idle warps
+constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
+constexpr uint32_t kTmemCols = 512;   // S0 | S1 | O0 | O1, 128 fp32 columns each
 constexpr long long kWaitCycles = 400000000ll;   // ~0.2 s at 2 GHz
+constexpr float kRescaleThreshold = 8.f;         // log2 units
 
 struct TcParams {
     const __nv_bfloat16* Q; __nv_bfloat16* O;
@@ -43,10 +57,8 @@ struct TcParams {
 
 // shared-memory map (dynamic, base aligned to 1024 B)
 constexpr int kOffQ = 0;
-constexpr int kOffK = kOffQ + kTileBytes;
-constexpr int kOffV = kOffK + kKvStages * kTileBytes;
-constexpr int kOffP = kOffV + kKvStages * kTileBytes;
-constexpr int kOffBar = kOffP + kTileBytes;
+constexpr int kOffRing = kOffQ + kQTiles * kTileBytes;
+constexpr int kOffBar = kOffRing + kStages * kTileBytes;
 constexpr int kSmemBytes = kOffBar + 256 + 1024;   // barriers + alignment slack
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -156,229 +168,269 @@ __device__ __forceinline__ uint32_t swz(int r, int cc) {
     return (uint32_t)((cc >> 3) * kHalfBytes + r * 128 + (((cc & 7) ^ (r & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kTileM, 1)
+
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int tile = gridDim.x - 1 - blockIdx.x;   // heaviest tiles first
+    const int pair = gridDim.x - 1 - blockIdx.x;   // heaviest row blocks first
     const int qh = blockIdx.y, b = blockIdx.z;
     const int nk = p.n_kept[b];
-    const int slot0 = tile * kTileM;
+    const int slot0 = pair * (kQTiles * kTileM);
     if (slot0 >= max(nk, 1)) return;
 
     const int32_t* kept = p.kept_idx + (size_t)b * p.S;
     __nv_bfloat16* Ob = p.O + (long long)b * p.os.b + (long long)qh * p.os.h;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     if (nk == 0) {   // nothing retained: the whole head is zero
-        for (int i = tid; i < p.S * 16; i += kTileM)
+        for (int i = tid; i < p.S * 16; i += kThreads)
             *reinterpret_cast<uint4*>(Ob + (long long)(i >> 4) * p.os.t + (i & 15) * 8) = zero4;
         return;
     }
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar_k = sbase + kOffBar, bar_v = bar_k + 16, bar_s = bar_v + 16, bar_o = bar_s + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 64);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar + 72);
+    const uint32_t bar_q = sbase + kOffBar;              // Q tiles written
+    const uint32_t bar_full = bar_q + 8;                 // [kStages] ring slot filled by TMA
+    const uint32_t bar_empty = bar_full + 8 * kStages;   // [kStages] ring slot consumed by the MMAs
+    const uint32_t bar_s = bar_empty + 8 * kStages;      // [2] S_i ready
+    const uint32_t bar_p = bar_s + 16;                   // [2] P_i written (and O_i rescaled)
+    const uint32_t bar_o = bar_p + 16;                   // all MMAs done
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 160);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar + 168);
 
-    // ---- this thread's row ------------------------------------------------------------------------
-    const int slot = slot0 + tid;
-    const bool valid = slot < nk;
-    const int t_row = valid ? kept[slot] : -1;
-    const int hi = t_row;
-    const int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
-    const int t_first = kept[slot0];
-    const int t_last = kept[min(slot0 + kTileM, nk) - 1];
-    const int j_begin = ((p.window > 0 ? max(0, t_first - p.window + 1) : 0) / kTileN) * kTileN;
-    const int n_tiles = (t_last - j_begin) / kTileN + 1;
+    // ---- which K/V tiles each Q tile needs (CTA-uniform) -------------------------------------------
+    int jb[kQTiles], je[kQTiles];
+#pragma unroll
+    for (int i = 0; i < kQTiles; ++i) {
+        const int s_lo = slot0 + i * kTileM;
+        if (s_lo < nk) {
+            const int t_first = kept[s_lo], t_last = kept[min(s_lo + kTileM, nk) - 1];
+            jb[i] = (p.window > 0 ? max(0, t_first - p.window + 1) : 0) / kTileN;
+            je[i] = t_last / kTileN + 1;
+        } else {
+            jb[i] = je[i] = 0;
+        }
+    }
+    const int n_q = (je[1] > jb[1]) ? 2 : 1;
+    const int J0 = jb[0], J1 = max(je[0], je[1]);   // rows ascend, so tile 0 starts first
     const int kh = qh / (p.Hq / p.Hkv);
 
     if (tid == 0) {
-        for (int i = 0; i < 2; ++i) { mbar_init(bar_k + 8 * i, 1); mbar_init(bar_v + 8 * i, 1); mbar_init(bar_s + 8 * i, 1); }
+        mbar_init(bar_q, n_q * kTileM);
+        for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, kTileM); }
         mbar_init(bar_o, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-
-    // ---- zero the rows of pruned tokens that precede this row (and follow the last retained one) ---
-    if (valid) {
-        const int prev = slot == 0 ? -1 : kept[slot - 1];
-        for (int t = prev + 1; t < t_row; ++t)
-            for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + c * 8) = zero4;
-        if (slot == nk - 1)
-            for (int t = t_row + 1; t < p.S; ++t)
-                for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + c * 8) = zero4;
-    }
-
-    // ---- gather Q rows into the swizzled K-major operand layout ---------------------------------
-    {
-        const __nv_bfloat16* qrow = p.Q + (long long)b * p.qs.b + (long long)max(t_row, 0) * p.qs.t + (long long)qh * p.qs.h;
-#pragma unroll
-        for (int cc = 0; cc < 16; ++cc) {
-            const uint4 v = valid ? ldg16(qrow + cc * 8) : zero4;
-            *reinterpret_cast<uint4*>(smem + kOffQ + swz(tid, cc)) = v;
-        }
-    }
-    fence_proxy_async();
+    if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 TMEM lanes
-    const uint32_t tm_o = tm_lane + 256;
 
-    auto load_k = [&](int it) {
-        const int st = it % kKvStages;
-        mbar_expect_tx(bar_k + 8 * st, kTileBytes);
-        tma_load_4d(sbase + kOffK + st * kTileBytes, &mapK, bar_k + 8 * st, 0, kh, j_begin + it * kTileN, b);
-        tma_load_4d(sbase + kOffK + st * kTileBytes + kHalfBytes, &mapK, bar_k + 8 * st, 64, kh, j_begin + it * kTileN, b);
-    };
-    auto load_v = [&](int it) {
-        const int st = it % kKvStages;
-        mbar_expect_tx(bar_v + 8 * st, kTileBytes);
-        tma_load_4d(sbase + kOffV + st * kTileBytes, &mapV, bar_v + 8 * st, 0, kh, j_begin + it * kTileN, b);
-        tma_load_4d(sbase + kOffV + st * kTileBytes + kHalfBytes, &mapV, bar_v + 8 * st, 64, kh, j_begin + it * kTileN, b);
-    };
-    auto issue_qk = [&](int it) {   // S[it % 2] = Q K[it]^T, 8 steps of 16 dims
-        const uint32_t kaddr = sbase + kOffK + (it % kKvStages) * kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-            mma_ss(tmem + (it & 1) * 128, desc_kmajor(sbase + kOffQ + off), desc_kmajor(kaddr + off), kIdescQK, kk > 0);
-        }
-        mma_commit(bar_s + 8 * (it & 1));
-    };
-    auto issue_pv = [&](int it) {   // O (+)= P V[it], 8 steps of 16 keys
-        const uint32_t vaddr = sbase + kOffV + (it % kKvStages) * kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t poff = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-            mma_ss(tmem + 256, desc_kmajor(sbase + kOffP + poff), desc_mnmajor(vaddr + kk * 16 * 128), kIdescPV,
-                   (it > 0 || kk > 0) ? 1u : 0u);
-        }
-        mma_commit(bar_o);
-    };
-
-    if (tid == 0) {
-        load_k(0); load_v(0);
-        if (n_tiles > 1) load_k(1);
-        mbar_wait(bar_k, 0, abort_flag, p.status, 1);
-        tc_fence_after();
-        issue_qk(0);
-    }
-    __syncwarp();
-
-    float m_run = -INFINITY, l_run = 0.f;
-    for (int it = 0; it < n_tiles; ++it) {
-        const int j0 = j_begin + it * kTileN;
-        // ---- S(it) is ready; get QK(it+1) going before the softmax ---------------------------------
-        mbar_wait(bar_s + 8 * (it & 1), (it >> 1) & 1, abort_flag, p.status, 2);
-        __syncwarp();
-        tc_fence_after();
-        if (tid == 0 && it + 1 < n_tiles) {
-            // K stage of tile it is free now (QK(it) done): fetch K(it+2) into it
-            if (it + 2 < n_tiles) load_k(it + 2);
-            mbar_wait(bar_k + 8 * ((it + 1) % kKvStages), ((it + 1) / kKvStages) & 1, abort_flag, p.status, 3);
-            tc_fence_after();
-            issue_qk(it + 1);
-        }
-        __syncwarp();   // the .sync.aligned TMEM accesses below need the whole warp together
-        // ---- softmax of row `tid` over the 128 keys of this tile ----------------------------------
-        uint32_t sreg[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tm_lane + (it & 1) * 128 + c * 32, sreg + c * 32);
-        tmem_wait_ld();
-        const bool full = (j0 >= lo) && (j0 + kTileN - 1 <= hi);
-        float mx = -INFINITY;
-        if (full) {
-#pragma unroll
-            for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
-        } else {
-#pragma unroll
-            for (int c = 0; c < 128; ++c) {
-                const int j = j0 + c;
-                const float s = (j >= lo && j <= hi) ? __uint_as_float(sreg[c]) : -INFINITY;
-                sreg[c] = __float_as_uint(s);
-                mx = fmaxf(mx, s);
+    // registers move from the third warpgroup (which needs few) to the two softmax groups
+    // (each setmaxnreg sits at the top of the branch it governs, so no later code sees both)
+    if (warp >= kMmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    if (warp == kTmaWarp) {
+        // ================================ TMA producer ================================================
+        if (lane == 0) {
+            int q = 0;
+            for (int j = J0; j < J1; ++j) {
+                for (int kv = 0; kv < 2; ++kv, ++q) {
+                    const int st = q % kStages;
+                    if (q >= kStages) mbar_wait(bar_empty + 8 * st, ((q / kStages) - 1) & 1, abort_flag, p.status, 10);
+                    const uint32_t dst = sbase + kOffRing + st * kTileBytes;
+                    const CUtensorMap* map = kv ? &mapV : &mapK;
+                    mbar_expect_tx(bar_full + 8 * st, kTileBytes);
+                    tma_load_4d(dst, map, bar_full + 8 * st, 0, kh, j * kTileN, b);
+                    tma_load_4d(dst + kHalfBytes, map, bar_full + 8 * st, 64, kh, j * kTileN, b);
+                }
             }
         }
-        const float m_new = fmaxf(m_run, mx * p.scale_log2);
-        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-        const float corr = ex2(m_run - m_safe);
-        float psum = 0.f;
-        uint32_t pk[64];
+    } else if (warp == kMmaWarp) {
+        // ================================ MMA issuer ==================================================
+        if (lane == 0) {
+            auto slot_of = [&](int j, int kv) { return (2 * (j - J0) + kv) % kStages; };
+            auto par_of = [&](int j, int kv) { return ((2 * (j - J0) + kv) / kStages) & 1; };
+            auto active = [&](int i, int j) { return j >= jb[i] && j < je[i]; };
+            auto issue_qk = [&](int i, int j) {   // S_i = Q_i K_j^T : 8 steps of 16 dims
+                const uint32_t kaddr = sbase + kOffRing + slot_of(j, 0) * kTileBytes;
+                const uint32_t qaddr = sbase + kOffQ + i * kTileBytes;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-            const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), p.scale_log2, -m_safe));
-            const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), p.scale_log2, -m_safe));
-            psum += p0 + p1;
-            pk[c] = pack_bf16(p0, p1);
-        }
-        l_run = fmaf(l_run, corr, psum);
-        m_run = m_new;
-
-        // ---- PV(it-1) must be complete before O is rescaled and P overwritten ---------------------
-        if (it > 0) {
-            mbar_wait(bar_o, (it - 1) & 1, abort_flag, p.status, 4);
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                    mma_ss(tmem + i * 128, desc_kmajor(qaddr + off), desc_kmajor(kaddr + off), kIdescQK, kk > 0);
+                }
+                mma_commit(bar_s + 8 * i);
+            };
+            auto issue_pv = [&](int i, int j, bool first) {   // O_i (+)= P_i V_j : 8 steps of 16 keys
+                const uint32_t vaddr = sbase + kOffRing + slot_of(j, 1) * kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, desc_mnmajor(vaddr + kk * 16 * 128), kIdescPV,
+                           (!first || kk > 0) ? 1u : 0u);
+            };
+            mbar_wait(bar_q, 0, abort_flag, p.status, 20);
+            mbar_wait(bar_full + 8 * slot_of(J0, 0), par_of(J0, 0), abort_flag, p.status, 21);
             tc_fence_after();
-            if (tid == 0 && it + 1 < n_tiles) load_v(it + 1);   // V stage of tile it-1 is free now
+            for (int i = 0; i < kQTiles; ++i)
+                if (active(i, J0)) issue_qk(i, J0);
+            mma_commit(bar_empty + 8 * slot_of(J0, 0));
+            int done[kQTiles] = {0, 0};
+            for (int j = J0; j < J1; ++j) {
+                mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.status, 22);
+                if (j + 1 < J1) mbar_wait(bar_full + 8 * slot_of(j + 1, 0), par_of(j + 1, 0), abort_flag, p.status, 23);
+#pragma unroll
+                for (int i = 0; i < kQTiles; ++i) {
+                    if (active(i, j)) {
+                        mbar_wait(bar_p + 8 * i, done[i] & 1, abort_flag, p.status, 24 + i);
+                        tc_fence_after();
+                        issue_pv(i, j, done[i] == 0);
+                        ++done[i];
+                    }
+                    if (i == kQTiles - 1) mma_commit(bar_empty + 8 * slot_of(j, 1));
+                    if (j + 1 < J1 && active(i, j + 1)) issue_qk(i, j + 1);
+                }
+                if (j + 1 < J1) mma_commit(bar_empty + 8 * slot_of(j + 1, 0));
+            }
+            mma_commit(bar_o);
+        }
+    }
+    } else {
+        // ================================ softmax groups ===============================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+        const int i = warp >> 2;                 // Q tile of this group
+        const int r = tid & (kTileM - 1);        // row within the tile
+        const int slot = slot0 + i * kTileM + r;
+        const bool valid = slot < nk;
+        const int t_row = valid ? kept[slot] : -1;
+        const int hi = t_row;
+        const int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
+        if (i < n_q) {
+            // gather this row of Q into the swizzled K-major operand layout
+            const __nv_bfloat16* qrow = p.Q + (long long)b * p.qs.b + (long long)max(t_row, 0) * p.qs.t + (long long)qh * p.qs.h;
+            uint4 qv[16];
+#pragma unroll
+            for (int cc = 0; cc < 16; ++cc) qv[cc] = valid ? ldg16(qrow + cc * 8) : zero4;
+#pragma unroll
+            for (int cc = 0; cc < 16; ++cc) *reinterpret_cast<uint4*>(smem + kOffQ + i * kTileBytes + swz(r, cc)) = qv[cc];
+            fence_proxy_async();
+            mbar_arrive(bar_q);
+        }
+        // rows of pruned tokens that precede this row (and follow the last retained one) are zero
+        if (valid) {
+            const int prev = slot == 0 ? -1 : kept[slot - 1];
+            for (int t = prev + 1; t < t_row; ++t)
+                for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + c * 8) = zero4;
+            if (slot == nk - 1)
+                for (int t = t_row + 1; t < p.S; ++t)
+                    for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + c * 8) = zero4;
+        }
+        __syncwarp();
+        const uint32_t tm_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + i * 128;   // this warp's lanes, S_i / P_i
+        const uint32_t tm_o = tm_s + 256;                                               // O_i
+        float m_ref = -INFINITY, l_run = 0.f;
+        for (int j = jb[i]; j < je[i]; ++j) {
+            const int c_it = j - jb[i];
+            const int j0 = j * kTileN;
+            mbar_wait(bar_s + 8 * i, c_it & 1, abort_flag, p.status, 30 + i);
             __syncwarp();
-            if (__any_sync(0xffffffffu, corr != 1.f)) {
+            tc_fence_after();
+            uint32_t sreg[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, sreg + c * 32);
+            tmem_wait_ld();
+            const bool full = (j0 >= lo) && (j0 + kTileN - 1 <= hi);
+            float mx = -INFINITY;
+            if (full) {
+#pragma unroll
+                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 128; ++c) {
+                    const int jj = j0 + c;
+                    const float s = (jj >= lo && jj <= hi) ? __uint_as_float(sreg[c]) : -INFINITY;
+                    sreg[c] = __float_as_uint(s);
+                    mx = fmaxf(mx, s);
+                }
+            }
+            __syncwarp();   // rows take different masking branches; the TMEM accesses below are warp-wide
+            // move the reference maximum only when the tile maximum exceeds it by 2^8 or more
+            const float m_tile = mx * p.scale_log2;
+            const bool move = m_tile > m_ref + kRescaleThreshold;   // also true on the first visible key (m_ref = -inf)
+            const float m_new = move ? m_tile : m_ref;
+            const float corr = move ? ex2(m_ref - m_new) : 1.f;
+            if (c_it > 0 && __any_sync(0xffffffffu, move)) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tm_o + c * 32, o);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * corr);
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * corr);
                     tmem_st32(tm_o + c * 32, o);
                 }
-                tmem_wait_st();
             }
-        } else if (tid == 0 && n_tiles > 1) {
-            load_v(1);
+            m_ref = m_new;
+            const float m_safe = (m_ref == -INFINITY) ? 0.f : m_ref;
+            float psum = 0.f;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const float p0 = ex2(fmaf(__uint_as_float(sreg[h * 64 + 2 * c]), p.scale_log2, -m_safe));
+                    const float p1 = ex2(fmaf(__uint_as_float(sreg[h * 64 + 2 * c + 1]), p.scale_log2, -m_safe));
+                    psum += p0 + p1;
+                    pk[c] = pack_bf16(p0, p1);
+                }
+                tmem_st32(tm_s + h * 32, pk);   // P_i over the first 64 columns of S_i
+            }
+            l_run = fmaf(l_run, corr, psum);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p + 8 * i);
         }
-#pragma unroll
-        for (int cc = 0; cc < 16; ++cc)
-            *reinterpret_cast<uint4*>(smem + kOffP + swz(tid, cc)) = make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+        // ---- epilogue: O / l -> bf16 -> the row's token position --------------------------------------
+        if (i < n_q) {
+            mbar_wait(bar_o, 0, abort_flag, p.status, 40);
+            __syncwarp();
             tc_fence_after();
-            mbar_wait(bar_v + 8 * (it % kKvStages), (it / kKvStages) & 1, abort_flag, p.status, 5);
-            tc_fence_after();
-            issue_pv(it);
-        }
-    }
-
-    // ---- epilogue: O / l -> bf16 -> the row's token position ------------------------------------
-    mbar_wait(bar_o, (n_tiles - 1) & 1, abort_flag, p.status, 6);
-    __syncwarp();
-    tc_fence_after();
-    {
-        const float inv = 1.f / l_run;
-        __nv_bfloat16* orow = Ob + (long long)max(t_row, 0) * p.os.t;
+            const float inv = 1.f / l_run;
+            __nv_bfloat16* orow = Ob + (long long)max(t_row, 0) * p.os.t;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tm_o + c * 32, o);
-            tmem_wait_ld();
-            if (valid) {
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tm_o + c * 32, o);
+                tmem_wait_ld();
+                if (valid) {
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    uint4 w;
-                    w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-                    w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-                    w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-                    w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                    *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    }
                 }
             }
         }
     }
+    __syncwarp();
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {   // a wait gave up: give copies and MMAs still in flight time to land before leaving
@@ -386,7 +438,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         while (clock64() - t0 < 2000000ll) { }
         __syncthreads();
     }
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ---- host side: tensor maps over the caller's K / V ----------------------------------------------
@@ -451,8 +503,9 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     tp.scale_log2 = scale * 1.4426950408889634f;
     tp.kept_idx = kept_idx; tp.n_kept = n_kept;
     tp.status = ctx->dev_status;
-    const dim3 grid((unsigned)((s.seq + kTileM - 1) / kTileM), (unsigned)s.n_q_heads, (unsigned)s.batch);
-    attention_tc_kernel<<<grid, kTileM, kSmemBytes, st>>>(tp, mapK, mapV);
+    const int rows_per_cta = kQTiles * kTileM;
+    const dim3 grid((unsigned)((s.seq + rows_per_cta - 1) / rows_per_cta), (unsigned)s.n_q_heads, (unsigned)s.batch);
+    attention_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tp, mapK, mapV);
     ctx->launches += 1;
     return cudaGetLastError();
 }
