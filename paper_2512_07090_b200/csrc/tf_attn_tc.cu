@@ -140,6 +140,30 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// packed fp32x2 arithmetic (two lanes per instruction) and the 3-input maximum
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t d;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -354,19 +378,21 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, sreg + c * 32);
             tmem_wait_ld();
             const bool full = (j0 >= lo) && (j0 + kTileN - 1 <= hi);
-            float mx = -INFINITY;
-            if (full) {
-#pragma unroll
-                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
-            } else {
+            if (!full) {
 #pragma unroll
                 for (int c = 0; c < 128; ++c) {
                     const int jj = j0 + c;
-                    const float s = (jj >= lo && jj <= hi) ? __uint_as_float(sreg[c]) : -INFINITY;
-                    sreg[c] = __float_as_uint(s);
-                    mx = fmaxf(mx, s);
+                    if (jj < lo || jj > hi) sreg[c] = 0xff800000u;   // -inf
                 }
             }
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains, not one of 128
+#pragma unroll
+            for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    mx4[u] = max3(mx4[u], __uint_as_float(sreg[c + 2 * u]), __uint_as_float(sreg[c + 2 * u + 1]));
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             __syncwarp();   // rows take different masking branches; the TMEM accesses below are warp-wide
             // move the reference maximum only when the tile maximum exceeds it by 2^8 or more
             const float m_tile = mx * p.scale_log2;
@@ -386,19 +412,25 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             }
             m_ref = m_new;
             const float m_safe = (m_ref == -INFINITY) ? 0.f : m_ref;
-            float psum = 0.f;
+            const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_safe, -m_safe);
+            uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t pk[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
-                    const float p0 = ex2(fmaf(__uint_as_float(sreg[h * 64 + 2 * c]), p.scale_log2, -m_safe));
-                    const float p1 = ex2(fmaf(__uint_as_float(sreg[h * 64 + 2 * c + 1]), p.scale_log2, -m_safe));
-                    psum += p0 + p1;
+                    float x0, x1;
+                    unpack2(fma2(pack2(__uint_as_float(sreg[h * 64 + 2 * c]), __uint_as_float(sreg[h * 64 + 2 * c + 1])), sc2, nm2), x0, x1);
+                    const float p0 = ex2(x0), p1 = ex2(x1);
+                    acc[c & 3] = add2(acc[c & 3], pack2(p0, p1));
                     pk[c] = pack_bf16(p0, p1);
                 }
                 tmem_st32(tm_s + h * 32, pk);   // P_i over the first 64 columns of S_i
             }
+            float a0, a1, a2, a3;
+            unpack2(add2(acc[0], acc[1]), a0, a1);
+            unpack2(add2(acc[2], acc[3]), a2, a3);
+            const float psum = (a0 + a1) + (a2 + a3);
             l_run = fmaf(l_run, corr, psum);
             tmem_wait_st();
             tc_fence_before();
