@@ -118,6 +118,34 @@ tf_status tf_kv_stats(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params
                       const void *K, const void *V, float *sim_k, float *sim_v,
                       const tf_carry *carry, void *stream);
 
+/* tf_kv_stats without any allocation on anybody's part.  (The paper has no counterpart to
+ * this entry; it exists for deployment only.)  Same inputs, outputs and arithmetic as
+ * tf_kv_stats, but the look-back records live in a fixed array of TF_STATIC_SCRATCH_BYTES that
+ * is built into the library, so no workspace has to be bound and no context is needed.  It is
+ * meant for callers that cannot obtain device memory at the point of the call: a server that
+ * has already given all free HBM to its KV-cache pool, code that must leave the device heap to
+ * a framework's caching allocator, or a latency-critical loop that cannot afford the
+ * device-wide stall of cudaMalloc / cudaFree.  The entry calls no cudaMalloc, cudaFree or
+ * other allocating routine.
+ *   - Runs on the CURRENT device.  ctx may be NULL; if given it must belong to the current
+ *     device, and device-side conditions (a wait that gave up) are recorded in it.  With NULL
+ *     they are not recorded anywhere.
+ *   - Limit: shapes whose records need more than TF_STATIC_SCRATCH_BYTES return
+ *     TF_ERR_WORKSPACE and launch nothing.  The records take 2 KiB per (64 tokens (bf16) or
+ *     32 tokens (fp32), sequence, KV head) plus one eighth of that; 8 MiB covers, for example,
+ *     batch 1 x 2048 tokens x 32 KV heads in bf16 three times over.
+ *   - The first call on each device looks up the array's device address and zeroes the part
+ *     it uses; make that first call outside any stream capture.
+ *   - Every GPU on which the library is loaded holds the array until the process exits.
+ *   - All calls in the process share the array of their device, and it keeps what the last
+ *     call left (stale records are recognised by their launch tag; the region is zeroed again
+ *     when the shape's record layout changes).  Two calls whose kernels overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them. */
+#define TF_STATIC_SCRATCH_BYTES (8u << 20)
+tf_status tf_kv_stats_static(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                             const void *K, const void *V, float *sim_k, float *sim_v,
+                             const tf_carry *carry, void *stream);
+
 /* Step a3 (Alg. 1 lines (s_k, sigma_k^2), alpha, s_KV; Eq. 2-3).  sim_k, sim_v fp32
  * [B,S,n_kv_heads] -> score fp32 [B,S].  Population variance over the KV heads. */
 tf_status tf_score_fuse(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,

@@ -23,9 +23,10 @@ TF_ANCHOR_PAST_MEAN, TF_ANCHOR_INCL_MEAN, TF_ANCHOR_EMA = 0, 1, 2
 TF_FUSE_INVVAR, TF_FUSE_EQ2_LITERAL, TF_FUSE_KEY_ONLY, TF_FUSE_VALUE_ONLY, TF_FUSE_MEAN = 0, 1, 2, 3, 4
 TF_SELECT_RATIO, TF_SELECT_THRESHOLD = 0, 1
 TF_KV_ALL, TF_KV_RETAINED = 0, 1
+TF_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
-           "tf_kv_stats", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
+           "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
            "tf_status_string")
 
@@ -159,6 +160,12 @@ class Context:
     def tf_kv_stats(self, shape, params, K, V, sim_k, sim_v, carry: Optional[tf_carry] = None):
         _check(lib().tf_kv_stats(self._h, C.byref(shape), C.byref(params), _ptr(K), _ptr(V), _ptr(sim_k),
                                  _ptr(sim_v), None if carry is None else C.byref(carry), _stream()), "tf_kv_stats")
+
+    def tf_kv_stats_static(self, shape, params, K, V, sim_k, sim_v, carry: Optional[tf_carry] = None):
+        """tf_kv_stats on the library's built-in scratch array: no workspace, nothing allocated."""
+        _check(lib().tf_kv_stats_static(self._h, C.byref(shape), C.byref(params), _ptr(K), _ptr(V), _ptr(sim_k),
+                                        _ptr(sim_v), None if carry is None else C.byref(carry), _stream()),
+               "tf_kv_stats_static")
 
     def tf_score_fuse(self, shape, params, sim_k, sim_v, score):
         _check(lib().tf_score_fuse(self._h, C.byref(shape), C.byref(params), _ptr(sim_k), _ptr(sim_v),
