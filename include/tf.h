@@ -192,8 +192,10 @@ tf_status tf_layer_filter_host(tf_ctx *ctx, const tf_shape *shape, const tf_filt
 tf_status tf_get_status(tf_ctx *ctx, int sync, int64_t detail[4]);
 tf_status tf_clear_status(tf_ctx *ctx);
 
-/* Which attention kernel a bf16 call uses: 1 = tcgen05 tensor-core kernel (default),
- * 0 = the plain CUDA-core kernel that fp32 always uses.  For A/B checks. */
+/* Which attention kernel a bf16 call uses: 1 = tcgen05 tensor-core kernel (default; it picks between
+ * its two work distributions by problem size), 0 = the plain CUDA-core kernel that fp32 always uses,
+ * 2 = tensor-core kernel, two Q tiles per CTA sharing every K/V tile, 3 = tensor-core kernel, one Q
+ * tile per CTA with its K/V tiles split between the CTA's two softmax groups.  For A/B checks. */
 tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
 
 const char *tf_status_string(tf_status s);

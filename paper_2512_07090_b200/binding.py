@@ -199,8 +199,9 @@ class Context:
     def tf_clear_status(self):
         _check(lib().tf_clear_status(self._h), "tf_clear_status")
 
-    def tf_set_attention_path(self, use_tensor_cores: bool):
-        _check(lib().tf_set_attention_path(self._h, C.c_int(1 if use_tensor_cores else 0)), "tf_set_attention_path")
+    def tf_set_attention_path(self, path):
+        """0 / False: CUDA-core kernel; 1 / True: tensor-core kernel (form chosen by size); 2: shared form; 3: split form."""
+        _check(lib().tf_set_attention_path(self._h, C.c_int(int(path))), "tf_set_attention_path")
 
     @property
     def launches(self) -> int:

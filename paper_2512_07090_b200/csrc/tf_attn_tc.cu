@@ -38,7 +38,6 @@ constexpr int kQTiles = 2;            // Q tiles per CTA
 constexpr int kTileN = 128;           // keys per K/V tile
 constexpr int kHalfBytes = 128 * 128; // one [128 rows][128 B] swizzled block (64 bf16 per row)
 constexpr int kTileBytes = 2 * kHalfBytes;
-constexpr int kStages = 4;            // ring slots, used K(j), V(j), K(j+1), V(j+1), ...
 constexpr int kSoftmaxThreads = kQTiles * kTileM;
 constexpr int kThreads = kSoftmaxThreads + 128;   // third warpgroup: MMA warp, TMA warp, two idle warps
 constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
@@ -53,13 +52,26 @@ struct TcParams {
     float scale_log2;
     const int32_t* kept_idx; const int32_t* n_kept;
     DevStatus* status;
+    int n_row_blocks;     // CTAs per (batch, query head)
+    int heads_fastest;    // CTA order: 1 = all heads of the heaviest row block first, 0 = all row blocks of a head together
 };
 
-// shared-memory map (dynamic, base aligned to 1024 B)
-constexpr int kOffQ = 0;
-constexpr int kOffRing = kOffQ + kQTiles * kTileBytes;
-constexpr int kOffBar = kOffRing + kStages * kTileBytes;
-constexpr int kSmemBytes = kOffBar + 256 + 1024;   // barriers + alignment slack
+// Two ways of giving the two softmax groups of a CTA their work:
+//   shared (kSplit = false): two consecutive 128-row Q tiles; every K/V tile is loaded once and used by both.
+//   split  (kSplit = true):  ONE 128-row Q tile; the groups take alternate K/V tiles and their partial
+//                            results (O, maximum, sum) are merged at the end.  Twice as many, half as
+//                            long CTAs: used when the shared form would leave SMs idle or unbalanced.
+template <bool kSplit> struct Cfg {
+    static constexpr int kQBufs = kSplit ? 1 : 2;         // Q tiles in shared memory
+    static constexpr int kStages = kSplit ? 6 : 4;        // ring slots, filled in the order K(j), V(j), K(j+1), V(j+1), ...
+    static constexpr int kRows = kQBufs * kTileM;         // retained rows per CTA
+    static constexpr int kStep = kSplit ? 2 : 1;          // K/V tile stride of one softmax group
+    // shared-memory map (dynamic, base aligned to 1024 B)
+    static constexpr int kOffQ = 0;
+    static constexpr int kOffRing = kOffQ + kQBufs * kTileBytes;
+    static constexpr int kOffBar = kOffRing + kStages * kTileBytes;
+    static constexpr int kSmemBytes = kOffBar + 256 + 1024;   // barriers + alignment slack
+};
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -202,14 +214,23 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
 }
 
+template <bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
+    using C = Cfg<kSplit>;
+    constexpr int kStages = C::kStages, kOffQ = C::kOffQ, kOffRing = C::kOffRing, kOffBar = C::kOffBar, kStep = C::kStep;
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pair = gridDim.x - 1 - blockIdx.x;   // heaviest row blocks first
-    const int qh = blockIdx.y, b = blockIdx.z;
+    // CTAs start in index order.  Row blocks of a head differ in length by the causal triangle, so the
+    // heaviest go first; with few CTAs per SM that has to hold across heads (heads_fastest), while a
+    // large problem keeps the row blocks of one head together so that they find its K/V in L2.
+    const int n_bh = (int)(gridDim.x / (unsigned)p.n_row_blocks);
+    const int rb = p.heads_fastest ? (int)blockIdx.x / n_bh : (int)blockIdx.x % p.n_row_blocks;
+    const int bh = p.heads_fastest ? (int)blockIdx.x % n_bh : (int)blockIdx.x / p.n_row_blocks;
+    const int pair = p.n_row_blocks - 1 - rb;
+    const int qh = bh % p.Hq, b = bh / p.Hq;
     const int nk = p.n_kept[b];
-    const int slot0 = pair * (kQTiles * kTileM);
+    const int slot0 = pair * C::kRows;
     if (slot0 >= max(nk, 1)) return;
 
     const int32_t* kept = p.kept_idx + (size_t)b * p.S;
@@ -233,24 +254,25 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar + 168);
 
     // ---- which K/V tiles each Q tile needs (CTA-uniform) -------------------------------------------
+    // group i works on tiles jb[i], jb[i] + kStep, ... < je[i]
     int jb[kQTiles], je[kQTiles];
 #pragma unroll
     for (int i = 0; i < kQTiles; ++i) {
-        const int s_lo = slot0 + i * kTileM;
+        const int s_lo = slot0 + (kSplit ? 0 : i * kTileM);
         if (s_lo < nk) {
             const int t_first = kept[s_lo], t_last = kept[min(s_lo + kTileM, nk) - 1];
-            jb[i] = (p.window > 0 ? max(0, t_first - p.window + 1) : 0) / kTileN;
+            jb[i] = (p.window > 0 ? max(0, t_first - p.window + 1) : 0) / kTileN + (kSplit ? i : 0);
             je[i] = t_last / kTileN + 1;
         } else {
             jb[i] = je[i] = 0;
         }
     }
-    const int n_q = (je[1] > jb[1]) ? 2 : 1;
+    const int n_q = kSplit ? 1 : ((je[1] > jb[1]) ? 2 : 1);   // Q tiles to gather
     const int J0 = jb[0], J1 = max(je[0], je[1]);   // rows ascend, so tile 0 starts first
     const int kh = qh / (p.Hq / p.Hkv);
 
     if (tid == 0) {
-        mbar_init(bar_q, n_q * kTileM);
+        mbar_init(bar_q, kSoftmaxThreads);
         for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, kTileM); }
         mbar_init(bar_o, 1);
@@ -268,7 +290,19 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     // (each setmaxnreg sits at the top of the branch it governs, so no later code sees both)
     if (warp >= kMmaWarp) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (warp == kTmaWarp) {
+    if (warp > kTmaWarp) {
+        // ================================ zero fill (the two spare warps) ================================
+        // rows of pruned tokens that precede a retained row of this CTA (and follow the last retained
+        // one) are zero; 16 lanes write one row
+        const int g4 = (tid - (kTmaWarp + 1) * 32) >> 4, l16 = tid & 15;
+        const int s_end = min(slot0 + C::kRows, nk);
+        for (int s_z = slot0 + g4; s_z < s_end; s_z += 4) {
+            const int prev = s_z == 0 ? -1 : kept[s_z - 1], cur = kept[s_z];
+            for (int t = prev + 1; t < cur; ++t) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + l16 * 8) = zero4;
+            if (s_z == nk - 1)
+                for (int t = cur + 1; t < p.S; ++t) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + l16 * 8) = zero4;
+        }
+    } else if (warp == kTmaWarp) {
         // ================================ TMA producer ================================================
         if (lane == 0) {
             int q = 0;
@@ -292,7 +326,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             auto active = [&](int i, int j) { return j >= jb[i] && j < je[i]; };
             auto issue_qk = [&](int i, int j) {   // S_i = Q_i K_j^T : 8 steps of 16 dims
                 const uint32_t kaddr = sbase + kOffRing + slot_of(j, 0) * kTileBytes;
-                const uint32_t qaddr = sbase + kOffQ + i * kTileBytes;
+                const uint32_t qaddr = sbase + kOffQ + (kSplit ? 0 : i) * kTileBytes;   // split: both groups share the Q tile
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
@@ -308,12 +342,35 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
                            (!first || kk > 0) ? 1u : 0u);
             };
             mbar_wait(bar_q, 0, abort_flag, p.status, 20);
+            int done[kQTiles] = {0, 0};
+            if constexpr (kSplit) {
+                // tile j belongs to group (j - J0) & 1; order: QK_0(J0), QK_1(J0+1), then per tile PV(j), QK(j+2)
+                for (int j = J0; j < min(J0 + 2, J1); ++j) {
+                    mbar_wait(bar_full + 8 * slot_of(j, 0), par_of(j, 0), abort_flag, p.status, 21);
+                    tc_fence_after();
+                    issue_qk(j - J0, j);
+                    mma_commit(bar_empty + 8 * slot_of(j, 0));
+                }
+                for (int j = J0; j < J1; ++j) {
+                    const int i = (j - J0) & 1;
+                    mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.status, 22);
+                    mbar_wait(bar_p + 8 * i, done[i] & 1, abort_flag, p.status, 24 + i);
+                    tc_fence_after();
+                    issue_pv(i, j, done[i] == 0);
+                    ++done[i];
+                    mma_commit(bar_empty + 8 * slot_of(j, 1));
+                    if (j + 2 < J1) {
+                        mbar_wait(bar_full + 8 * slot_of(j + 2, 0), par_of(j + 2, 0), abort_flag, p.status, 23);
+                        issue_qk(i, j + 2);
+                        mma_commit(bar_empty + 8 * slot_of(j + 2, 0));
+                    }
+                }
+            } else {
             mbar_wait(bar_full + 8 * slot_of(J0, 0), par_of(J0, 0), abort_flag, p.status, 21);
             tc_fence_after();
             for (int i = 0; i < kQTiles; ++i)
                 if (active(i, J0)) issue_qk(i, J0);
             mma_commit(bar_empty + 8 * slot_of(J0, 0));
-            int done[kQTiles] = {0, 0};
             for (int j = J0; j < J1; ++j) {
                 mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.status, 22);
                 if (j + 1 < J1) mbar_wait(bar_full + 8 * slot_of(j + 1, 0), par_of(j + 1, 0), abort_flag, p.status, 23);
@@ -330,45 +387,49 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
                 }
                 if (j + 1 < J1) mma_commit(bar_empty + 8 * slot_of(j + 1, 0));
             }
+            }
             mma_commit(bar_o);
         }
     }
     } else {
         // ================================ softmax groups ===============================================
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-        const int i = warp >> 2;                 // Q tile of this group
+        const int i = warp >> 2;                 // group: its Q tile (shared) or its half of the K/V tiles (split)
         const int r = tid & (kTileM - 1);        // row within the tile
-        const int slot = slot0 + i * kTileM + r;
+        const int slot = slot0 + (kSplit ? 0 : i * kTileM) + r;
         const bool valid = slot < nk;
         const int t_row = valid ? kept[slot] : -1;
         const int hi = t_row;
         const int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
-        if (i < n_q) {
-            // gather this row of Q into the swizzled K-major operand layout
-            const __nv_bfloat16* qrow = p.Q + (long long)b * p.qs.b + (long long)max(t_row, 0) * p.qs.t + (long long)qh * p.qs.h;
-            uint4 qv[16];
+        {
+            // gather the CTA's Q rows into the swizzled K-major operand layout: 16 lanes fetch one row
+            // (256 contiguous bytes), the 8 warps take 16 rows per round
+            constexpr int kRounds = C::kRows / 16;
+            const int sub = lane >> 4, cc = lane & 15, w8 = tid >> 5;
+            int tq[kRounds];
 #pragma unroll
-            for (int cc = 0; cc < 16; ++cc) qv[cc] = valid ? ldg16(qrow + cc * 8) : zero4;
+            for (int it = 0; it < kRounds; ++it) {
+                const int s_q = slot0 + it * 16 + w8 * 2 + sub;
+                tq[it] = s_q < nk ? kept[s_q] : -1;
+            }
+            uint4 qv[kRounds];
+            const __nv_bfloat16* qbase = p.Q + (long long)b * p.qs.b + (long long)qh * p.qs.h + cc * 8;
 #pragma unroll
-            for (int cc = 0; cc < 16; ++cc) *reinterpret_cast<uint4*>(smem + kOffQ + i * kTileBytes + swz(r, cc)) = qv[cc];
+            for (int it = 0; it < kRounds; ++it) qv[it] = tq[it] >= 0 ? ldg16(qbase + (long long)tq[it] * p.qs.t) : zero4;
+#pragma unroll
+            for (int it = 0; it < kRounds; ++it) {
+                const int rr = it * 16 + w8 * 2 + sub;
+                *reinterpret_cast<uint4*>(smem + kOffQ + (rr >> 7) * kTileBytes + swz(rr & (kTileM - 1), cc)) = qv[it];
+            }
             fence_proxy_async();
             mbar_arrive(bar_q);
-        }
-        // rows of pruned tokens that precede this row (and follow the last retained one) are zero
-        if (valid) {
-            const int prev = slot == 0 ? -1 : kept[slot - 1];
-            for (int t = prev + 1; t < t_row; ++t)
-                for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + c * 8) = zero4;
-            if (slot == nk - 1)
-                for (int t = t_row + 1; t < p.S; ++t)
-                    for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + c * 8) = zero4;
         }
         __syncwarp();
         const uint32_t tm_s = tmem + ((uint32_t)((warp & 3) * 32) << 16) + i * 128;   // this warp's lanes, S_i / P_i
         const uint32_t tm_o = tm_s + 256;                                               // O_i
         float m_ref = -INFINITY, l_run = 0.f;
-        for (int j = jb[i]; j < je[i]; ++j) {
-            const int c_it = j - jb[i];
+        for (int j = jb[i]; j < je[i]; j += kStep) {
+            const int c_it = (j - jb[i]) / kStep;
             const int j0 = j * kTileN;
             mbar_wait(bar_s + 8 * i, c_it & 1, abort_flag, p.status, 30 + i);
             __syncwarp();
@@ -378,11 +439,17 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, sreg + c * 32);
             tmem_wait_ld();
             const bool full = (j0 >= lo) && (j0 + kTileN - 1 <= hi);
-            if (!full) {
+            if (!full) {   // columns below c_lo or above c_hi are invisible to this row: -inf
+                const int c_lo = lo - j0, c_hi = hi - j0;
+                if (c_lo <= 0) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c) {
-                    const int jj = j0 + c;
-                    if (jj < lo || jj > hi) sreg[c] = 0xff800000u;   // -inf
+                    for (int c = 0; c < 128; ++c) if (c > c_hi) sreg[c] = 0xff800000u;
+                } else if (c_hi >= kTileN - 1) {
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) if (c < c_lo) sreg[c] = 0xff800000u;
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 128; ++c) if (c < c_lo || c > c_hi) sreg[c] = 0xff800000u;
                 }
             }
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains, not one of 128
@@ -437,7 +504,49 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             mbar_arrive(bar_p + 8 * i);
         }
         // ---- epilogue: O / l -> bf16 -> the row's token position --------------------------------------
-        if (i < n_q) {
+        if constexpr (kSplit) {
+            // merge the two groups' partial results: both accumulators sit in the TMEM lanes of this row,
+            // so each group finishes 64 of the 128 output columns; (maximum, sum) travel through the
+            // shared memory of the Q tile, which nobody reads once every MMA has completed
+            mbar_wait(bar_o, 0, abort_flag, p.status, 40);
+            __syncwarp();
+            tc_fence_after();
+            float2* ml = reinterpret_cast<float2*>(smem + kOffQ);
+            ml[i * kTileM + r] = make_float2(m_ref, l_run);
+            asm volatile("bar.sync 1, %0;" :: "n"(kSoftmaxThreads) : "memory");
+            const float2 other = ml[(i ^ 1) * kTileM + r];
+            const bool both = je[1] > jb[1];                       // group 1 had tiles (CTA-uniform)
+            const float m0 = i == 0 ? m_ref : other.x, l0 = i == 0 ? l_run : other.y;   // group 0 always has a tile
+            const float m1 = i == 0 ? other.x : m_ref, l1 = i == 0 ? other.y : l_run;
+            const float m_all = both ? fmaxf(m0, m1) : m0;
+            const float e0 = ex2(m0 - m_all), e1 = both ? ex2(m1 - m_all) : 0.f;
+            const float inv = 1.f / (l0 * e0 + l1 * e1);
+            const float w0 = e0 * inv, w1 = e1 * inv;
+            const uint32_t tm_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+            __nv_bfloat16* orow = Ob + (long long)max(t_row, 0) * p.os.t + i * 64;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t o0[32], o1[32];
+                tmem_ld32(tm_row + 256 + i * 64 + c * 32, o0);
+                if (both) tmem_ld32(tm_row + 384 + i * 64 + c * 32, o1);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        float f[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            f[e] = __uint_as_float(o0[8 * v + e]) * w0;
+                            if (both) f[e] = fmaf(__uint_as_float(o1[8 * v + e]), w1, f[e]);
+                        }
+                        uint4 w;
+                        w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
+                        w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    }
+                }
+            }
+        } else if (i < n_q) {
             mbar_wait(bar_o, 0, abort_flag, p.status, 40);
             __syncwarp();
             tc_fence_after();
@@ -512,7 +621,6 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
                                 const void* Q, const void* K, const void* V,
                                 const int32_t* kept_idx, const int32_t* n_kept, void* O,
                                 cudaStream_t st) {
-    (void)p;
     if (s.dtype != TF_BF16 || s.head_dim != kHeadDim) return cudaErrorNotSupported;
     if (s.batch == 0 || s.seq == 0) return cudaSuccess;
     CUtensorMap mapK, mapV;
@@ -521,7 +629,11 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         return cudaErrorNotSupported;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Cfg<false>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg<true>::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -535,9 +647,22 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     tp.scale_log2 = scale * 1.4426950408889634f;
     tp.kept_idx = kept_idx; tp.n_kept = n_kept;
     tp.status = ctx->dev_status;
-    const int rows_per_cta = kQTiles * kTileM;
-    const dim3 grid((unsigned)((s.seq + rows_per_cta - 1) / rows_per_cta), (unsigned)s.n_q_heads, (unsigned)s.batch);
-    attention_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tp, mapK, mapV);
+    // The shared form needs enough CTAs to fill and balance the SMs (CTAs of one head differ in length by
+    // the causal triangle); below that the split form, with twice as many CTAs of half the length, wins.
+    // The number of retained rows is only known on the device: the ratio gives the expected count.
+    const double kept_frac = (p.select_mode == TF_SELECT_RATIO) ? 1.0 - p.prune_ratio : 1.0;
+    const double ctas_shared = (double)s.batch * s.n_q_heads * ceil(s.seq * kept_frac / (kQTiles * kTileM));
+    int sms = 148;
+    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+    const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 0.75 * sms);
+    const int rows_per_cta = split ? kTileM : kQTiles * kTileM;
+    tp.n_row_blocks = (s.seq + rows_per_cta - 1) / rows_per_cta;
+    const double kv_bytes = 2.0 * s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
+    tp.heads_fastest = (kv_bytes <= 48e6 || ctas_shared < 6.0 * sms) ? 1 : 0;   // K and V stay in L2, or balance matters more
+    const long long n_ctas = (long long)tp.n_row_blocks * s.n_q_heads * s.batch;
+    if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
+    if (split) attention_tc_kernel<true><<<(unsigned)n_ctas, kThreads, Cfg<true>::kSmemBytes, st>>>(tp, mapK, mapV);
+    else       attention_tc_kernel<false><<<(unsigned)n_ctas, kThreads, Cfg<false>::kSmemBytes, st>>>(tp, mapK, mapV);
     ctx->launches += 1;
     return cudaGetLastError();
 }

@@ -95,6 +95,7 @@ struct tf_ctx {
     tf::ScanScratch scan_user;     // scan bookkeeping of the caller's workspace
     tf::ScanScratch scan_owned;    // ... and of owned_ws
     int use_tensor_cores;          // bf16 attention path
+    int attention_form;            // tensor-core kernel: 0 = choose by grid size, 1 = shared K/V tiles, 2 = split K/V tiles
     long long launches;            // kernels launched through this context
     // tf_layer_filter_host staging (owned, grown on demand)
     void* stage;

@@ -155,7 +155,9 @@ def test_select_bit_exact_ties_eligibility_nan_threshold(case):
 
 
 # ------------------------------------------------------------------------------- a5
-@pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, True), (torch.bfloat16, False), (torch.float32, False)])
+# path 2 / 3: the tensor-core kernel with K/V tiles shared by two Q tiles / split between the softmax groups
+@pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 1),
+                                                (torch.bfloat16, 0), (torch.float32, 0)])
 @pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5),
                                                     (1, 257, 8, 2, 0, 0.3), (2, 300, 4, 1, 64, 0.5),
                                                     (1, 515, 2, 2, 1, 0.7), (1, 200, 4, 2, 0, 0.99),
@@ -177,9 +179,11 @@ def test_pruned_attention_matches_oracle(dtype, tensor_cores, B, S, Hq, Hkv, win
     g.close()
 
 
-def test_pruned_attention_nothing_kept_and_everything_kept():
+@pytest.mark.parametrize("path", [2, 3])
+def test_pruned_attention_nothing_kept_and_everything_kept(path):
     q, k, v = _qkv(2, 70, 2, 2, torch.bfloat16)
     g = Gpu(q, k, v)
+    g.ctx.tf_set_attention_path(path)
     idx = torch.full((2, 70), -1, dtype=torch.int32, device=DEV)
     idx[1] = torch.arange(70, dtype=torch.int32, device=DEV)
     nk = torch.tensor([0, 70], dtype=torch.int32, device=DEV)
