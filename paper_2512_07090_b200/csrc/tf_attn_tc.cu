@@ -221,6 +221,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     constexpr int kStages = C::kStages, kOffQ = C::kOffQ, kOffRing = C::kOffRing, kOffBar = C::kOffBar, kStep = C::kStep;
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    grid_dependency_wait();   // kept_idx / n_kept come from the kernel before this one
     // CTAs start in index order.  Row blocks of a head differ in length by the causal triangle, so the
     // heaviest go first; with few CTAs per SM that has to hold across heads (heads_fastest), while a
     // large problem keeps the row blocks of one head together so that they find its K/V in L2.
@@ -661,10 +662,11 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     tp.heads_fastest = (kv_bytes <= 48e6 || ctas_shared < 6.0 * sms) ? 1 : 0;   // K and V stay in L2, or balance matters more
     const long long n_ctas = (long long)tp.n_row_blocks * s.n_q_heads * s.batch;
     if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
-    if (split) attention_tc_kernel<true><<<(unsigned)n_ctas, kThreads, Cfg<true>::kSmemBytes, st>>>(tp, mapK, mapV);
-    else       attention_tc_kernel<false><<<(unsigned)n_ctas, kThreads, Cfg<false>::kSmemBytes, st>>>(tp, mapK, mapV);
+    cudaError_t e;
+    if (split) e = launch_dependent(attention_tc_kernel<true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<true>::kSmemBytes, st, tp, mapK, mapV);
+    else       e = launch_dependent(attention_tc_kernel<false>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace tf

@@ -73,6 +73,22 @@ __device__ __forceinline__ float warp_max(float v) {
 // ---- host-side launch bookkeeping --------------------------------------------------------------
 struct Strides3 { long long b, t, h; };
 
+// Launch a kernel that may start while the kernel before it on the stream drains (programmatic
+// dependent launch).  Such a kernel executes grid_dependency_wait() before it touches global memory;
+// until then only its launch and set-up overlap with its predecessor.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 }  // namespace tf
 
 namespace tf {

@@ -365,6 +365,7 @@ __global__ void __launch_bounds__(256) score_fuse_kernel(const float* __restrict
                                                          const float* __restrict__ sim_v,
                                                          float* __restrict__ score, long long n_tokens,
                                                          int H, int mode, float eps, DevStatus* status) {
+    grid_dependency_wait();
     const long long tok = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (tok >= n_tokens) return;
@@ -409,10 +410,10 @@ cudaError_t launch_score_fuse(tf_ctx* ctx, const tf_shape& s, const tf_filter_pa
     const float eps = p.var_eps > 0.f ? p.var_eps : 1e-8f;
     const long long threads = n * 32;
     const unsigned blocks = (unsigned)((threads + 255) / 256);
-    score_fuse_kernel<<<blocks, 256, 0, st>>>(sim_k, sim_v, score, n, s.n_kv_heads, p.fuse_mode, eps,
-                                              ctx->dev_status);
+    cudaError_t e = launch_dependent(score_fuse_kernel, dim3(blocks), dim3(256), 0, st, sim_k, sim_v, score, n,
+                                     s.n_kv_heads, p.fuse_mode, eps, ctx->dev_status);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace tf

@@ -61,6 +61,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     __shared__ unsigned int s_prefix;
     __shared__ int s_rank, s_count;
 
+    grid_dependency_wait();
     const int b = blockIdx.x, tid = threadIdx.x, S = p.S;
     const float* sc = p.score + (size_t)b * S;
     const uint8_t* el = p.eligible ? p.eligible + (size_t)b * S : nullptr;
@@ -202,9 +203,9 @@ cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params
     sp.S = s.seq; sp.warmup = p.warmup_tokens; sp.mode = p.select_mode;
     sp.p_target = (long long)floor(p.prune_ratio * (double)s.seq);
     sp.keep_mask = keep_mask; sp.kept_idx = kept_idx; sp.n_kept = n_kept; sp.theta = theta;
-    select_kernel<<<s.batch, kSelThreads, 0, st>>>(sp);
+    cudaError_t e = launch_dependent(select_kernel, dim3(s.batch), dim3(kSelThreads), 0, st, sp);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace tf
