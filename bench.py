@@ -271,27 +271,42 @@ def main():
     ms = e0.elapsed_time(e1)
     launches = ctx.launches - l0
 
-    # ---- per-kernel durations: the same steps through the four stage entry points -----------------
+    # ---- per-kernel durations: each stage entry point alone, K launches back to back ---------------
+    # (events around the whole loop, so launch latency is not charged to the kernel; every ring entry
+    #  first gets its own similarities / scores / kept list from one pass through the stages)
     names = ("kv_stats", "score_fuse", "select", "pruned_attention")
     per = {n: 0.0 for n in names}
     flops = 0.0
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
-    for i in range(args.steps):
-        q, k, v = ring[(args.warmup + i) % len(ring)]
-        ev = evs[i]
-        ev[0].record(); ctx.tf_kv_stats(shape, params, k, v, sim_k, sim_v)
-        ev[1].record(); ctx.tf_score_fuse(shape, params, sim_k, sim_v, score)
-        ev[2].record(); ctx.tf_select(shape, params, score, keep, idx, nk)
-        ev[3].record(); ctx.tf_pruned_attention(shape, params, q, k, v, idx, nk, O)
-        ev[4].record()
-        if i < len(ring):
-            torch.cuda.synchronize()
-            flops += attention_flops(idx.cpu().numpy(), nk.cpu().numpy(), Hq, d, wl.window)
-    torch.cuda.synchronize()
-    flops /= min(args.steps, len(ring))
-    for ev in evs:
-        for j, n in enumerate(names):
-            per[n] += ev[j].elapsed_time(ev[j + 1]) / args.steps
+    state = []
+    for q, k, v in ring:
+        sk, sv = torch.empty_like(sim_k), torch.empty_like(sim_v)
+        sc, ix, n_ = torch.empty_like(score), torch.empty_like(idx), torch.empty_like(nk)
+        ctx.tf_kv_stats(shape, params, k, v, sk, sv)
+        ctx.tf_score_fuse(shape, params, sk, sv, sc)
+        ctx.tf_select(shape, params, sc, keep, ix, n_)
+        torch.cuda.synchronize()
+        flops += attention_flops(ix.cpu().numpy(), n_.cpu().numpy(), Hq, d, wl.window) / len(ring)
+        state.append((sk, sv, sc, ix, n_))
+
+    def stage(name, i):
+        q, k, v = ring[i % len(ring)]
+        sk, sv, sc, ix, n_ = state[i % len(ring)]
+        if name == "kv_stats": ctx.tf_kv_stats(shape, params, k, v, sim_k, sim_v)
+        elif name == "score_fuse": ctx.tf_score_fuse(shape, params, sk, sv, score)
+        elif name == "select": ctx.tf_select(shape, params, sc, keep, idx, nk)
+        else: ctx.tf_pruned_attention(shape, params, q, k, v, ix, n_, O)
+
+    for n in names:
+        for i in range(3):
+            stage(n, i)
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for i in range(args.steps):
+            stage(n, args.warmup + i)
+        s1.record()
+        torch.cuda.synchronize()
+        per[n] = s0.elapsed_time(s1) / args.steps
     clocks = sampler.stop()
 
     if dist is not None:

@@ -186,6 +186,16 @@ tf_status tf_layer_filter_host(tf_ctx *ctx, const tf_shape *shape, const tf_filt
                                void *O_host, float *score_host, uint8_t *keep_mask_host,
                                int32_t *kept_idx_host, int32_t *n_kept_host, void *stream);
 
+/* Tail-focused layer policy (Section 3.3, "P_tail = P_global / Y").  Host-only helper: fills
+ * ratio_per_layer[0 .. n_layers) (HOST memory) with the pruning ratio each layer should be run
+ * at so that the whole stack meets the global budget: the last n_tail = round(tail_fraction *
+ * n_layers) layers (at least one) get p_global / tail_fraction, all earlier layers get 0 (they
+ * are not filtered at all, so they pay no scoring overhead).  n_tail_out (may be NULL) receives
+ * n_tail.  TF_ERR_INVALID_ARG if a ratio is outside [0,1), tail_fraction outside (0,1], or the
+ * per-layer ratio would reach 1. */
+tf_status tf_tail_policy(double p_global, double tail_fraction, int32_t n_layers,
+                         double *ratio_per_layer, int32_t *n_tail_out);
+
 /* Device-side conditions since the last tf_clear_status: returns TF_OK, TF_ERR_TIMEOUT or
  * TF_ERR_NAN_SCORE.  sync != 0 synchronises the device first.  detail (may be NULL) receives
  * four words: {code, where, count of NaN scores, kernels launched by this context}. */

@@ -168,3 +168,10 @@ def layer_filter(Q, K, V, prune_ratio=0.5, warmup_tokens=1, eligible=None, windo
     if attention:
         out["O"] = pruned_attention(Q, K, V, sel["keep_mask"], window, scale, kv_visibility)
     return out
+
+
+def tail_policy(p_global, tail_fraction, n_layers):
+    """Section 3.3: only the last round(Y * n_layers) layers are filtered, each at P_tail = P_global / Y
+    (the paper's equation for P_tail); earlier layers are not filtered.  Returns the per-layer ratios."""
+    n_tail = min(n_layers, max(1, int(np.floor(tail_fraction * n_layers + 0.5))))
+    return [p_global / tail_fraction if l >= n_layers - n_tail else 0.0 for l in range(n_layers)]

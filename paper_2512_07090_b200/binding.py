@@ -28,7 +28,7 @@ TF_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
-           "tf_status_string")
+           "tf_status_string", "tf_tail_policy")
 
 
 class tf_shape(C.Structure):
@@ -118,6 +118,15 @@ def make_shape(Q: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, O: O
         getattr(s, name)[:] = [t.stride(0), t.stride(1), t.stride(2)]
     s.window, s.softmax_scale = int(window), float(softmax_scale)
     return s
+
+
+def tail_policy(p_global: float, tail_fraction: float, n_layers: int):
+    """Per-layer pruning ratios of the tail-focused policy (host helper); returns (ratios, n_tail)."""
+    out = (C.c_double * n_layers)()
+    n_tail = C.c_int32()
+    _check(lib().tf_tail_policy(C.c_double(p_global), C.c_double(tail_fraction), C.c_int32(n_layers), out,
+                                C.byref(n_tail)), "tf_tail_policy")
+    return list(out), int(n_tail.value)
 
 
 class Context:

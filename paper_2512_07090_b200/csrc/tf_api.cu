@@ -320,6 +320,20 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
     return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
 }
 
+tf_status tf_tail_policy(double p_global, double tail_fraction, int32_t n_layers, double* ratio_per_layer,
+                         int32_t* n_tail_out) {
+    if (!ratio_per_layer || n_layers <= 0) return TF_ERR_INVALID_ARG;
+    if (!(p_global >= 0.0 && p_global < 1.0) || !(tail_fraction > 0.0 && tail_fraction <= 1.0)) return TF_ERR_INVALID_ARG;
+    const double p_tail = p_global / tail_fraction;
+    if (!(p_tail < 1.0)) return TF_ERR_INVALID_ARG;
+    int n_tail = (int)floor(tail_fraction * (double)n_layers + 0.5);
+    if (n_tail < 1) n_tail = 1;
+    if (n_tail > n_layers) n_tail = n_layers;
+    for (int l = 0; l < n_layers; ++l) ratio_per_layer[l] = (l >= n_layers - n_tail) ? p_tail : 0.0;
+    if (n_tail_out) *n_tail_out = n_tail;
+    return TF_OK;
+}
+
 tf_status tf_get_status(tf_ctx* ctx, int sync, int64_t detail[4]) {
     if (!ctx) return TF_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);

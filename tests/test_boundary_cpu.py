@@ -86,3 +86,15 @@ def test_no_cpu_fallback_exists():
         tfb.LIB_PATH, tfb._lib = path, saved
     src = open(os.path.join(ROOT, "paper_2512_07090_b200", "binding.py")).read()
     assert "import oracle" not in src and "from oracle" not in src
+
+
+def test_tail_policy_matches_the_oracle_and_rejects_bad_input(L):
+    import oracle
+    for pg, y, n in [(0.25, 0.5, 32), (0.2, 0.4, 40), (0.33, 0.6, 40), (0.1, 1.0, 7), (0.3, 0.37, 13)]:
+        got, n_tail = tfb.tail_policy(pg, y, n)
+        ref = oracle.tail_policy(pg, y, n)
+        assert got == ref and n_tail == sum(1 for x in ref if x > 0)
+    out = (C.c_double * 4)()
+    for pg, y, n in [(0.6, 0.5, 4), (-0.1, 0.5, 4), (0.2, 0.0, 4), (0.2, 1.5, 4), (0.2, 0.5, 0)]:
+        assert L.tf_tail_policy(C.c_double(pg), C.c_double(y), C.c_int32(n), out, None) == tfb.TF_ERR_INVALID_ARG
+    assert L.tf_tail_policy(C.c_double(0.2), C.c_double(0.5), C.c_int32(4), None, None) == tfb.TF_ERR_INVALID_ARG

@@ -353,3 +353,15 @@ def test_layer_filter_end_to_end_invariants():
     # GQA: statistics over KV heads == statistics over the g-fold expanded heads
     r2 = orc.layer_filter(q, np.repeat(k, 4, 2), np.repeat(v, 4, 2), prune_ratio=0.5, warmup_tokens=4)
     assert np.allclose(r2["score"], r["score"], atol=1e-13) and np.allclose(r2["O"], r["O"], atol=1e-12)
+
+
+# ------------------------------------------------------------------------------- tail-focused policy
+def test_tail_policy_paper_example_and_budget():
+    """Section 3.3's worked example: global budget 25 %, last half of the layers => 50 % per tail layer;
+    the mean over all layers is the global budget whenever Y * n_layers is whole."""
+    r = orc.tail_policy(0.25, 0.5, 32)
+    assert r[:16] == [0.0] * 16 and all(abs(x - 0.5) < 1e-15 for x in r[16:])
+    for pg, y, L in [(0.25, 0.5, 32), (0.2, 0.4, 40), (0.33, 0.6, 40), (0.1, 1.0, 7)]:
+        r = orc.tail_policy(pg, y, L)
+        assert abs(sum(r) / L - pg) < 1e-12
+        assert all(x == 0.0 for x in r[: L - round(y * L)])
