@@ -186,6 +186,36 @@ tf_status tf_layer_filter_host(tf_ctx *ctx, const tf_shape *shape, const tf_filt
                                void *O_host, float *score_host, uint8_t *keep_mask_host,
                                int32_t *kept_idx_host, int32_t *n_kept_host, void *stream);
 
+/* State of the online decode step, per sequence, all DEVICE memory owned by the caller:
+ * sum_k, sum_v fp32 [B, n_kv_heads, 128]: sums of the keys / values seen so far (EMA mode: the anchors
+ * of Eq. 1); count [B]: tokens in them; tau fp32 [B]: the layer's skip threshold; steps, skips [B]:
+ * decisions made and skips decided so far (their ratio is the running skip ratio).  sum_k, sum_v and
+ * count have the layout of tf_carry, so a prefill's tf_kv_stats can fill them (sum_*_out, count = S). */
+typedef struct {
+    float *sum_k, *sum_v;
+    int64_t *count;
+    float *tau;
+    int64_t *steps, *skips;
+} tf_decode_state;
+
+/* One decoding iteration of one layer (Algorithm 1 as printed, one new token per sequence): cosine of
+ * the current token's key / value to the anchors in `state`, (mean, var) over heads, alpha, s_KV;
+ * threshold adaptation tau += eta * (skip ratio so far - params->prune_ratio)   (Section 3.3,
+ * "T_l <- T_l + eta (P_current - P_tail)"; alg1_sign != 0 uses Algorithm 1's printed sign instead);
+ * the token skips attention iff s_KV > tau and pos >= params->warmup_tokens (decisions inside the
+ * warm-up still count toward the ratio); the anchors take the token in; unless skipped, the token's
+ * attention output is computed against cache positions <= pos (shape->window applies), else it is 0.
+ *   shape: batch, n_q_heads, n_kv_heads, dtype; seq = capacity of the caches; k_stride / v_stride
+ *          address K_cache / V_cache [B, seq, n_kv_heads, 128]; q_stride[0], q_stride[2] are the batch
+ *          and head strides of q_new [B, n_q_heads, 128], o_stride[0], o_stride[2] those of O_new.
+ *   pos:   device int32 [B], 0 <= pos[b] < seq, the cache row that already holds the current token.
+ *   score (may be NULL) fp32 [B]; skip u8 [B] (required): 1 = attention skipped, O_new row is zero.
+ * Two launches on the stream; the state is advanced in place. */
+tf_status tf_decode_step(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                         float eta, int32_t alg1_sign, const void *q_new, const void *K_cache,
+                         const void *V_cache, const int32_t *pos, const tf_decode_state *state,
+                         void *O_new, float *score, uint8_t *skip, void *stream);
+
 /* Tail-focused layer policy (Section 3.3, "P_tail = P_global / Y").  Host-only helper: fills
  * ratio_per_layer[0 .. n_layers) (HOST memory) with the pruning ratio each layer should be run
  * at so that the whole stack meets the global budget: the last n_tail = round(tail_fraction *

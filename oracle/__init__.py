@@ -175,3 +175,78 @@ def tail_policy(p_global, tail_fraction, n_layers):
     (the paper's equation for P_tail); earlier layers are not filtered.  Returns the per-layer ratios."""
     n_tail = min(n_layers, max(1, int(np.floor(tail_fraction * n_layers + 0.5))))
     return [p_global / tail_fraction if l >= n_layers - n_tail else 0.0 for l in range(n_layers)]
+
+
+# ---------------------------------------------------------------------------------------------------
+# Online decode step (Algorithm 1 as a per-token procedure, with the threshold feedback of Section 3.3)
+# ---------------------------------------------------------------------------------------------------
+def decode_state(B, Hkv, d=128, tau0=0.0):
+    """Empty per-sequence state: anchor sums, token count, threshold, decisions made, skips decided."""
+    return dict(sum_k=np.zeros((B, Hkv, d)), sum_v=np.zeros((B, Hkv, d)), count=np.zeros(B, np.int64),
+                tau=np.full(B, float(tau0)), steps=np.zeros(B, np.int64), skips=np.zeros(B, np.int64))
+
+
+def _cos_to_anchor(x, anchor, has_past):
+    """cosine of each head's vector to its anchor, each norm clamped at 1e-8; 0 where there is no past."""
+    num = (x * anchor).sum(-1)
+    den = np.maximum(np.sqrt((x * x).sum(-1)), 1e-8) * np.maximum(np.sqrt((anchor * anchor).sum(-1)), 1e-8)
+    return np.where(has_past, num / den, 0.0)
+
+
+def decode_step(state, q, K_cache, V_cache, pos, target_ratio=0.5, eta=0.05, warmup_tokens=1,
+                anchor_mode=ANCHOR_PAST_MEAN, gamma=0.9, fuse_mode=FUSE_INVVAR, var_eps=1e-8,
+                window=0, scale=0.0, alg1_sign=False):
+    """One decoding iteration of one layer for B sequences, in the order of Algorithm 1:
+    anchors -> per-head cosine of the current token's key / value -> (mean, var) over heads -> alpha ->
+    s_KV -> threshold adaptation -> skip decision; then the anchor takes the current token in, and the
+    attention of the current token (query q against cache positions <= pos) is computed unless skipped
+    (a skipped token's attention output is zero).
+
+    Threshold adaptation: tau += eta * (rho - target)   (Section 3.3, T_l += eta (P_current - P_tail)),
+    rho = skips decided / decisions made so far (0 before the first); alg1_sign=True uses the sign
+    printed in Algorithm 1, eta * (target - rho).  A token at position < warmup_tokens is never
+    skipped, but its decision still counts toward rho (the thresholds keep adapting during warm-up).
+
+    q [B,Hq,d], K_cache / V_cache [B,S,Hkv,d] with the current token already stored at pos[b].
+    state is updated in place.  Returns dict(score [B], skip [B] uint8, tau [B] after the update, O [B,Hq,d])."""
+    q = np.asarray(q, np.float64); K = np.asarray(K_cache, np.float64); V = np.asarray(V_cache, np.float64)
+    B, S, Hkv, d = K.shape
+    Hq = q.shape[1]
+    pos = np.asarray(pos, np.int64)
+    score = np.zeros(B); skip = np.zeros(B, np.uint8); O = np.zeros((B, Hq, d))
+    for b in range(B):
+        k, v = K[b, pos[b]], V[b, pos[b]]                      # [Hkv, d]
+        n = int(state["count"][b])
+        upd = (lambda s_, x: gamma * s_ + (1 - gamma) * x) if anchor_mode == ANCHOR_EMA else (lambda s_, x: s_ + x)
+        if anchor_mode == ANCHOR_INCL_MEAN:                    # anchor takes the current token in first
+            state["sum_k"][b] = upd(state["sum_k"][b], k); state["sum_v"][b] = upd(state["sum_v"][b], v)
+            n += 1
+        has_past = n > 0
+        div = 1.0 if anchor_mode == ANCHOR_EMA else max(n, 1)
+        ck = _cos_to_anchor(k, state["sum_k"][b] / div, has_past)
+        cv = _cos_to_anchor(v, state["sum_v"][b] / div, has_past)
+        s = float(score_fuse(ck[None, None, :], cv[None, None, :], fuse_mode, var_eps)[0, 0])
+        steps, skips = int(state["steps"][b]), int(state["skips"][b])
+        rho = skips / steps if steps > 0 else 0.0
+        e32, t32 = float(np.float32(eta)), float(np.float32(target_ratio))   # the kernel holds these two in fp32
+        delta = e32 * ((t32 - rho) if alg1_sign else (rho - t32))
+        state["tau"][b] = np.float32(np.float32(state["tau"][b]) + np.float32(delta))   # the threshold is kept in fp32
+        decide = bool(np.float32(s) > state["tau"][b]) if s == s else False
+        do_skip = decide and pos[b] >= warmup_tokens
+        state["steps"][b] = steps + 1
+        state["skips"][b] = skips + (1 if decide else 0)
+        if anchor_mode != ANCHOR_INCL_MEAN:
+            state["sum_k"][b] = upd(state["sum_k"][b], k); state["sum_v"][b] = upd(state["sum_v"][b], v)
+            n += 1
+        state["count"][b] = n
+        score[b] = s; skip[b] = 1 if do_skip else 0
+        if not do_skip:
+            g = Hq // Hkv
+            sc = scale if scale else 1.0 / np.sqrt(d)
+            lo = max(0, int(pos[b]) - window + 1) if window > 0 else 0
+            for h in range(Hq):
+                kk = K[b, lo:pos[b] + 1, h // g]; vv = V[b, lo:pos[b] + 1, h // g]
+                a = sc * (kk @ q[b, h])
+                a = np.exp(a - a.max())
+                O[b, h] = (a / a.sum()) @ vv
+    return dict(score=score, skip=skip, tau=state["tau"].copy(), O=O)

@@ -28,7 +28,7 @@ TF_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
-           "tf_status_string", "tf_tail_policy")
+           "tf_status_string", "tf_tail_policy", "tf_decode_step")
 
 
 class tf_shape(C.Structure):
@@ -49,6 +49,11 @@ class tf_filter_params(C.Structure):
 class tf_carry(C.Structure):
     _fields_ = [("sum_k_in", C.c_void_p), ("sum_v_in", C.c_void_p), ("count_in", C.c_void_p),
                 ("sum_k_out", C.c_void_p), ("sum_v_out", C.c_void_p)]
+
+
+class tf_decode_state(C.Structure):
+    _fields_ = [("sum_k", C.c_void_p), ("sum_v", C.c_void_p), ("count", C.c_void_p),
+                ("tau", C.c_void_p), ("steps", C.c_void_p), ("skips", C.c_void_p)]
 
 
 class TokenFilterError(RuntimeError):
@@ -129,6 +134,20 @@ def tail_policy(p_global: float, tail_fraction: float, n_layers: int):
     return list(out), int(n_tail.value)
 
 
+class DecodeState:
+    """Device tensors of the decode-step state and the struct that points at them."""
+
+    def __init__(self, B: int, Hkv: int, device, tau0: float = 0.0):
+        self.sum_k = torch.zeros(B, Hkv, 128, device=device)
+        self.sum_v = torch.zeros(B, Hkv, 128, device=device)
+        self.count = torch.zeros(B, dtype=torch.int64, device=device)
+        self.tau = torch.full((B,), float(tau0), device=device)
+        self.steps = torch.zeros(B, dtype=torch.int64, device=device)
+        self.skips = torch.zeros(B, dtype=torch.int64, device=device)
+        self.struct = tf_decode_state(*(t.data_ptr() for t in (self.sum_k, self.sum_v, self.count, self.tau,
+                                                               self.steps, self.skips)))
+
+
 class Context:
     """Owns a tf_ctx and (optionally) a torch-allocated workspace bound to it."""
 
@@ -192,6 +211,13 @@ class Context:
         _check(lib().tf_layer_filter(self._h, C.byref(shape), C.byref(params), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
                                      _ptr(score), _ptr(keep_mask), _ptr(kept_idx), _ptr(n_kept), _stream()),
                "tf_layer_filter")
+
+    def tf_decode_step(self, shape, params, eta, q_new, K_cache, V_cache, pos, state: "DecodeState", O_new,
+                       score=None, skip=None, alg1_sign=False):
+        _check(lib().tf_decode_step(self._h, C.byref(shape), C.byref(params), C.c_float(eta),
+                                    C.c_int32(1 if alg1_sign else 0), _ptr(q_new), _ptr(K_cache), _ptr(V_cache),
+                                    _ptr(pos), C.byref(state.struct), _ptr(O_new), _ptr(score), _ptr(skip), _stream()),
+               "tf_decode_step")
 
     def tf_layer_filter_host(self, shape, params, Q, K, V, O, score=None, keep_mask=None, kept_idx=None, n_kept=None):
         """Host tensors in, host tensors out (copies inside the call; returns after the stream is idle)."""

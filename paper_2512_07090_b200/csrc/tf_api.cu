@@ -14,10 +14,10 @@ inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 // Sections of the caller's workspace.
 struct WsLayout {
-    size_t scan, sim_k, sim_v, score, keep_mask, kept_idx, n_kept, theta, total;
+    size_t scan, sim_k, sim_v, score, keep_mask, kept_idx, n_kept, theta, kv_compact, total;
 };
 
-WsLayout ws_layout(const tf_shape& s) {
+WsLayout ws_layout(const tf_shape& s, const tf_filter_params* p) {
     WsLayout w{};
     const size_t tokens = (size_t)s.batch * (size_t)s.seq;
     size_t off = 0;
@@ -29,6 +29,8 @@ WsLayout ws_layout(const tf_shape& s) {
     w.kept_idx = off;  off += align256(tokens * sizeof(int32_t));
     w.n_kept = off;    off += align256((size_t)s.batch * sizeof(int32_t));
     w.theta = off;     off += align256((size_t)s.batch * sizeof(float));
+    w.kv_compact = off;   // retained tokens' K and V (TF_KV_RETAINED on the tensor-core path only)
+    if (p && p->kv_visibility == TF_KV_RETAINED && s.dtype == TF_BF16) off += kv_compact_bytes(s);
     w.total = off;
     return w;
 }
@@ -87,10 +89,16 @@ struct DeviceGuard {
 tf_status attention_dispatch(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const void* Q,
                              const void* K, const void* V, const int32_t* kept_idx,
                              const int32_t* n_kept, void* O, cudaStream_t st) {
-    if (p.kv_visibility != TF_KV_ALL) return TF_ERR_UNSUPPORTED;
     cudaError_t e = cudaErrorNotSupported;
-    if (s.dtype == TF_BF16 && ctx->use_tensor_cores)
-        e = launch_attention_tc(ctx, s, p, Q, K, V, kept_idx, n_kept, O, st);
+    if (s.dtype == TF_BF16 && ctx->use_tensor_cores) {
+        void* kv_compact = nullptr;
+        if (p.kv_visibility == TF_KV_RETAINED) {   // needs the workspace section for the retained K / V
+            const WsLayout w = ws_layout(s, &p);
+            if (!ctx->workspace || ctx->workspace_bytes < w.total) return TF_ERR_WORKSPACE;
+            kv_compact = static_cast<char*>(ctx->workspace) + w.kv_compact;
+        }
+        e = launch_attention_tc(ctx, s, p, Q, K, V, kept_idx, n_kept, O, kv_compact, st);
+    }
     if (e == cudaErrorNotSupported) e = launch_attention_simt(ctx, s, p, Q, K, V, kept_idx, n_kept, O, st);
     return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
 }
@@ -143,11 +151,10 @@ tf_status tf_destroy(tf_ctx* ctx) {
 }
 
 tf_status tf_workspace_bytes(const tf_shape* shape, const tf_filter_params* params, size_t* bytes) {
-    (void)params;
     if (!bytes) return TF_ERR_INVALID_ARG;
     tf_status s = check_shape(shape);
     if (s != TF_OK) return s;
-    *bytes = ws_layout(*shape).total;
+    *bytes = ws_layout(*shape, params).total;
     return TF_OK;
 }
 
@@ -234,8 +241,7 @@ tf_status tf_layer_filter(tf_ctx* ctx, const tf_shape* shape, const tf_filter_pa
     if (!Q || !O) return TF_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(O)) return TF_ERR_UNSUPPORTED;
     if (!stride_ok(shape->q_stride, shape->dtype) || !stride_ok(shape->o_stride, shape->dtype)) return TF_ERR_UNSUPPORTED;
-    if (params->kv_visibility != TF_KV_ALL) return TF_ERR_UNSUPPORTED;
-    const WsLayout w = ws_layout(*shape);
+    const WsLayout w = ws_layout(*shape, params);
     if (!ctx->workspace || ctx->workspace_bytes < w.total) return TF_ERR_WORKSPACE;
     DeviceGuard g(ctx->device);
     if (!g.ok) return TF_ERR_CUDA;
@@ -288,7 +294,7 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         if (cudaMalloc(&ctx->stage, need) != cudaSuccess) return TF_ERR_CUDA;
         ctx->stage_bytes = need;
     }
-    const WsLayout w = ws_layout(*shape);
+    const WsLayout w = ws_layout(*shape, params);
     if (ctx->owned_ws_bytes < w.total) {
         if (ctx->owned_ws) { cudaStreamSynchronize(st); cudaFree(ctx->owned_ws); ctx->owned_ws = nullptr; ctx->owned_ws_bytes = 0; }
         if (cudaMalloc(&ctx->owned_ws, w.total) != cudaSuccess) return TF_ERR_CUDA;
@@ -317,6 +323,28 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
     if (e == cudaSuccess && kept_idx_host) e = cudaMemcpyAsync(kept_idx_host, dI, tokens * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && n_kept_host) e = cudaMemcpyAsync(n_kept_host, dN, (size_t)shape->batch * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+}
+
+tf_status tf_decode_step(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params, float eta,
+                         int32_t alg1_sign, const void* q_new, const void* K_cache, const void* V_cache,
+                         const int32_t* pos, const tf_decode_state* state, void* O_new, float* score,
+                         uint8_t* skip, void* stream) {
+    if (!ctx) return TF_ERR_INVALID_ARG;
+    tf_status s = check_shape(shape);
+    if (s == TF_OK) s = check_params(params);
+    if (s == TF_OK) s = check_kv(shape, K_cache, V_cache);
+    if (s != TF_OK) return s;
+    if (!q_new || !O_new || !pos || !skip || !state) return TF_ERR_INVALID_ARG;
+    if (!state->sum_k || !state->sum_v || !state->count || !state->tau || !state->steps || !state->skips)
+        return TF_ERR_INVALID_ARG;
+    if (!(eta >= 0.f)) return TF_ERR_INVALID_ARG;
+    if (params->kv_visibility != TF_KV_ALL) return TF_ERR_UNSUPPORTED;
+    if (shape->q_stride[2] <= 0 || shape->o_stride[2] <= 0) return TF_ERR_UNSUPPORTED;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return TF_ERR_CUDA;
+    tf::tf_decode_args a{q_new, K_cache, V_cache, pos, state, O_new, score, skip, eta, alg1_sign ? 1 : 0};
+    cudaError_t e = launch_decode_step(ctx, *shape, *params, a, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
 }
 

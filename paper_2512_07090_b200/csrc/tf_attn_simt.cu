@@ -20,6 +20,7 @@ struct AttnParams {
     float scale_log2;          // softmax scale * log2(e)
     const int32_t* kept_idx;   // [B,S]
     const int32_t* n_kept;     // [B]
+    int retained_only;         // 1: a retained query sees retained tokens' keys / values only
 };
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
@@ -66,13 +67,18 @@ __global__ void __launch_bounds__(kSimtWarps * 32) attention_simt_kernel(const A
     for (int i = 0; i < 4; ++i) q_s[warp][lane * 4 + i] = to_f<T>(qrow[lane * 4 + i]) * p.scale_log2;
     __syncwarp();
 
-    const int j_lo = (p.window > 0) ? max(0, t - p.window + 1) : 0;
+    // keys are visited by index: token positions, or positions in the retained list (retained_only),
+    // where entry c stands for token kept[c] and the query itself is entry `slot`
+    const int t_min = (p.window > 0) ? max(0, t - p.window + 1) : 0;
+    const int j_hi = p.retained_only ? slot : t;
+    const int j_lo = p.retained_only ? first_kept_at_or_after(kept, slot + 1, t_min) : t_min;
     float m = -1e30f, lsum = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int j0 = j_lo; j0 <= t; j0 += 32) {
+    for (int j0 = j_lo; j0 <= j_hi; j0 += 32) {
         const int j = j0 + lane;
         float s = -1e30f;
-        if (j <= t) {
-            const T* krow = Kb + (long long)j * p.ks.t;
+        const int tok = (j <= j_hi) ? (p.retained_only ? kept[j] : j) : 0;
+        if (j <= j_hi) {
+            const T* krow = Kb + (long long)tok * p.ks.t;
             float d0 = 0.f, d1 = 0.f;
 #pragma unroll 4
             for (int v = 0; v < NVEC; ++v) {
@@ -86,14 +92,15 @@ __global__ void __launch_bounds__(kSimtWarps * 32) attention_simt_kernel(const A
         }
         const float m_new = fmaxf(m, warp_max(s));
         const float corr = exp2f(m - m_new);
-        const float pj = (j <= t) ? exp2f(s - m_new) : 0.f;
+        const float pj = (j <= j_hi) ? exp2f(s - m_new) : 0.f;
         lsum = lsum * corr + warp_sum(pj);
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[i] *= corr;
-        const int n_here = min(32, t - j0 + 1);
+        const int n_here = min(32, j_hi - j0 + 1);
         for (int jj = 0; jj < n_here; ++jj) {
             const float pw = __shfl_sync(0xffffffffu, pj, jj);
-            const T* vrow = Vb + (long long)(j0 + jj) * p.vs.t + lane * 4;
+            const int vt = __shfl_sync(0xffffffffu, tok, jj);
+            const T* vrow = Vb + (long long)vt * p.vs.t + lane * 4;
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[i] = fmaf(pw, to_f<T>(vrow[i]), acc[i]);
         }
@@ -109,9 +116,9 @@ cudaError_t launch_attention_simt(tf_ctx* ctx, const tf_shape& s, const tf_filte
                                   const void* Q, const void* K, const void* V,
                                   const int32_t* kept_idx, const int32_t* n_kept, void* O,
                                   cudaStream_t st) {
-    (void)p;
     if (s.batch == 0 || s.seq == 0) return cudaSuccess;
     AttnParams ap{};
+    ap.retained_only = (p.kv_visibility == TF_KV_RETAINED);
     ap.Q = Q; ap.K = K; ap.V = V; ap.O = O;
     ap.qs = {s.q_stride[0], s.q_stride[1], s.q_stride[2]};
     ap.ks = {s.k_stride[0], s.k_stride[1], s.k_stride[2]};

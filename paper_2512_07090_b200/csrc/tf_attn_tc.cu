@@ -28,6 +28,8 @@
 // stops waiting, lets copies in flight land, releases its TMEM and exits.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "tf_common.cuh"
 
 namespace tf {
@@ -52,6 +54,7 @@ struct TcParams {
     float scale_log2;
     const int32_t* kept_idx; const int32_t* n_kept;
     DevStatus* status;
+    int compact;          // 1: K / V hold the retained tokens only, entry c = token kept_idx[c] (TF_KV_RETAINED)
     int n_row_blocks;     // CTAs per (batch, query head)
     int heads_fastest;    // CTA order: 1 = all heads of the heaviest row block first, 0 = all row blocks of a head together
 };
@@ -261,9 +264,16 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     for (int i = 0; i < kQTiles; ++i) {
         const int s_lo = slot0 + (kSplit ? 0 : i * kTileM);
         if (s_lo < nk) {
-            const int t_first = kept[s_lo], t_last = kept[min(s_lo + kTileM, nk) - 1];
-            jb[i] = (p.window > 0 ? max(0, t_first - p.window + 1) : 0) / kTileN + (kSplit ? i : 0);
-            je[i] = t_last / kTileN + 1;
+            const int s_last = min(s_lo + kTileM, nk) - 1;
+            const int t_first = kept[s_lo], t_last = kept[s_last];
+            int k_first = p.window > 0 ? max(0, t_first - p.window + 1) : 0;   // first key the tile's first row sees
+            int k_last = t_last;                                                // last key its last row sees
+            if (p.compact) {   // keys are entries of the retained list
+                k_first = p.window > 0 ? first_kept_at_or_after(kept, s_lo + 1, k_first) : 0;
+                k_last = s_last;
+            }
+            jb[i] = k_first / kTileN + (kSplit ? i : 0);
+            je[i] = k_last / kTileN + 1;
         } else {
             jb[i] = je[i] = 0;
         }
@@ -400,8 +410,12 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         const int slot = slot0 + (kSplit ? 0 : i * kTileM) + r;
         const bool valid = slot < nk;
         const int t_row = valid ? kept[slot] : -1;
-        const int hi = t_row;
-        const int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
+        int hi = t_row;                                                           // visible keys: lo .. hi
+        int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
+        if (p.compact && valid) {
+            lo = p.window > 0 ? first_kept_at_or_after(kept, slot + 1, lo) : 0;
+            hi = slot;
+        }
         {
             // gather the CTA's Q rows into the swizzled K-major operand layout: 16 lanes fetch one row
             // (256 contiguous bytes), the 8 warps take 16 rows per round
@@ -616,17 +630,66 @@ bool make_kv_map(CUtensorMap* map, const void* base, const int64_t st[3], int B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// TF_KV_RETAINED: copy the retained tokens' K and V rows (all KV heads) to dense [B,S,Hkv,128] buffers,
+// entry c of a sequence = token kept_idx[c]; entries from n_kept up to the next multiple of the key tile
+// are zeroed (they are masked, but a tile may not contain NaN bit patterns: 0 * NaN would reach O).
+__global__ void __launch_bounds__(256) compact_kv_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+                                                         Strides3 ks, Strides3 vs, int S, int Hkv,
+                                                         const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ n_kept,
+                                                         __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc) {
+    grid_dependency_wait();
+    const int b = blockIdx.y, nk = n_kept[b];
+    const int c_end = min(S, (nk + kTileN - 1) / kTileN * kTileN);
+    const int chunks = Hkv * 16;                               // 16-byte chunks per row of one tensor
+    const int32_t* kept = kept_idx + (size_t)b * S;
+    for (int c = blockIdx.x * 8 + (threadIdx.x >> 5); c < c_end; c += gridDim.x * 8) {
+        const bool live = c < nk;
+        const long long t = live ? kept[c] : 0;
+        for (int q = threadIdx.x & 31; q < chunks; q += 32) {
+            const int h = q >> 4, off = (q & 15) * 8;
+            uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+            if (live) {
+                kv = ldg16(K + (long long)b * ks.b + t * ks.t + (long long)h * ks.h + off);
+                vv = ldg16(V + (long long)b * vs.b + t * vs.t + (long long)h * vs.h + off);
+            }
+            const size_t dst = (((size_t)b * S + c) * Hkv + h) * kHeadDim + off;
+            *reinterpret_cast<uint4*>(Kc + dst) = kv;
+            *reinterpret_cast<uint4*>(Vc + dst) = vv;
+        }
+    }
+}
+
 }  // namespace
+
+size_t kv_compact_bytes(const tf_shape& s) {
+    return 2 * ((size_t)s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16) + 255) / 256 * 256;
+}
 
 cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                                 const void* Q, const void* K, const void* V,
                                 const int32_t* kept_idx, const int32_t* n_kept, void* O,
-                                cudaStream_t st) {
+                                void* kv_compact, cudaStream_t st) {
     if (s.dtype != TF_BF16 || s.head_dim != kHeadDim) return cudaErrorNotSupported;
     if (s.batch == 0 || s.seq == 0) return cudaSuccess;
+    const bool compact = (p.kv_visibility == TF_KV_RETAINED);
     CUtensorMap mapK, mapV;
-    if (!make_kv_map(&mapK, K, s.k_stride, s.batch, s.seq, s.n_kv_heads) ||
-        !make_kv_map(&mapV, V, s.v_stride, s.batch, s.seq, s.n_kv_heads))
+    if (compact) {
+        if (!kv_compact) return cudaErrorNotSupported;
+        __nv_bfloat16* Kc = static_cast<__nv_bfloat16*>(kv_compact);
+        __nv_bfloat16* Vc = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(kv_compact) + kv_compact_bytes(s) / 2);
+        const int64_t dense[3] = {(int64_t)s.seq * s.n_kv_heads * kHeadDim, (int64_t)s.n_kv_heads * kHeadDim, kHeadDim};
+        if (!make_kv_map(&mapK, Kc, dense, s.batch, s.seq, s.n_kv_heads) ||
+            !make_kv_map(&mapV, Vc, dense, s.batch, s.seq, s.n_kv_heads))
+            return cudaErrorNotSupported;
+        const Strides3 ks = {s.k_stride[0], s.k_stride[1], s.k_stride[2]}, vs = {s.v_stride[0], s.v_stride[1], s.v_stride[2]};
+        const unsigned gx = (unsigned)std::min<long long>(((long long)s.seq + 7) / 8, 4096);
+        cudaError_t e = launch_dependent(compact_kv_kernel, dim3(gx, (unsigned)s.batch), dim3(256), 0, st,
+                                         static_cast<const __nv_bfloat16*>(K), static_cast<const __nv_bfloat16*>(V), ks, vs,
+                                         s.seq, s.n_kv_heads, kept_idx, n_kept, Kc, Vc);
+        ctx->launches += 1;
+        if (e != cudaSuccess) return e;
+    } else if (!make_kv_map(&mapK, K, s.k_stride, s.batch, s.seq, s.n_kv_heads) ||
+               !make_kv_map(&mapV, V, s.v_stride, s.batch, s.seq, s.n_kv_heads))
         return cudaErrorNotSupported;
     static bool attr_set = false;
     if (!attr_set) {
@@ -648,6 +711,7 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     tp.scale_log2 = scale * 1.4426950408889634f;
     tp.kept_idx = kept_idx; tp.n_kept = n_kept;
     tp.status = ctx->dev_status;
+    tp.compact = compact ? 1 : 0;
     // The shared form needs enough CTAs to fill and balance the SMs (CTAs of one head differ in length by
     // the causal triangle); below that the split form, with twice as many CTAs of half the length, wins.
     // The number of retained rows is only known on the device: the ratio gives the expected count.

@@ -70,6 +70,16 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
+// first index c in the ascending list kept[0..n) with kept[c] >= target (n if none)
+__device__ __forceinline__ int first_kept_at_or_after(const int32_t* kept, int n, int target) {
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (kept[mid] < target) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
 // ---- host-side launch bookkeeping --------------------------------------------------------------
 struct Strides3 { long long b, t, h; };
 
@@ -144,10 +154,20 @@ cudaError_t launch_attention_simt(tf_ctx* ctx, const tf_shape& s, const tf_filte
                                   const void* Q, const void* K, const void* V,
                                   const int32_t* kept_idx, const int32_t* n_kept, void* O,
                                   cudaStream_t st);
+struct tf_decode_args {
+    const void* q_new; const void* K_cache; const void* V_cache; const int32_t* pos;
+    const tf_decode_state* state; void* O_new; float* score_out; uint8_t* skip_out;
+    float eta; int alg1_sign;
+};
+cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const tf_decode_args& a,
+                               cudaStream_t st);
 // returns cudaErrorNotSupported when the tensor-core path cannot take this call
+// kv_compact: TF_KV_RETAINED only -- device scratch of kv_compact_bytes(s) bytes for the retained
+// tokens' keys and values
 cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                                 const void* Q, const void* K, const void* V,
                                 const int32_t* kept_idx, const int32_t* n_kept, void* O,
-                                cudaStream_t st);
+                                void* kv_compact, cudaStream_t st);
+size_t kv_compact_bytes(const tf_shape& s);
 
 }  // namespace tf

@@ -179,6 +179,39 @@ def test_pruned_attention_matches_oracle(dtype, tensor_cores, B, S, Hq, Hkv, win
     g.close()
 
 
+@pytest.mark.parametrize("dtype,path", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 0), (torch.float32, 0)])
+@pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5), (1, 257, 8, 2, 0, 0.3),
+                                                    (2, 300, 4, 1, 64, 0.5), (1, 515, 2, 2, 1, 0.7),
+                                                    (1, 1300, 4, 2, 300, 0.5), (2, 1024, 2, 1, 0, 0.25)])
+def test_pruned_attention_retained_keys_only(dtype, path, B, S, Hq, Hkv, window, ratio):
+    """TF_KV_RETAINED: a retained query attends to retained tokens only (a pruned token's key and value
+    are gone for later queries as well); the window still counts original positions."""
+    q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=S + 1)
+    qn, kn, vn = oracle_inputs(q, k, v)
+    ref = oracle.layer_filter(qn, kn, vn, prune_ratio=ratio, warmup_tokens=1, window=window,
+                              kv_visibility=oracle.KV_RETAINED)
+    g = Gpu(q, k, v, window=window, kv_visibility=tfb.TF_KV_RETAINED)
+    g.ctx.tf_set_attention_path(path)
+    idx = torch.from_numpy(ref["kept_idx"]).to(DEV)
+    nk = torch.from_numpy(ref["n_kept"]).to(DEV)
+    g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
+    g.status_ok()
+    o = to_np(g.O)
+    assert np.isfinite(o).all()
+    assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
+    assert np.all(o[ref["keep_mask"] == 0] == 0.0)
+    if ratio > 0 and S > 100 and window == 0:   # and it is a different function from the all-keys reading
+        dense = oracle.layer_filter(qn, kn, vn, prune_ratio=ratio, warmup_tokens=1, window=window)
+        assert attn_rel_err(dense["O"], ref["O"]) > 10 * ATTN_TOL[dtype]
+    g.close()
+
+
+def test_layer_filter_retained_keys_only():
+    q, k, v = _qkv(2, 700, 8, 2, torch.bfloat16, seed=77)
+    n_mis = _layer_case(q, k, v, window=0, prune_ratio=0.5, warmup_tokens=4, kv_visibility=tfb.TF_KV_RETAINED)
+    assert n_mis == 0
+
+
 @pytest.mark.parametrize("path", [2, 3])
 def test_pruned_attention_nothing_kept_and_everything_kept(path):
     q, k, v = _qkv(2, 70, 2, 2, torch.bfloat16)
@@ -272,3 +305,64 @@ def test_device_rejects_bad_arguments_without_launching():
                          None, st) == tfb.TF_ERR_WORKSPACE
     assert g.ctx.launches == n0
     g.close()
+
+
+# ------------------------------------------------------------------------------- online decode step
+@pytest.mark.parametrize("dtype,mode,window", [(torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0), (torch.float32, tfb.TF_ANCHOR_PAST_MEAN, 40),
+                                               (torch.bfloat16, tfb.TF_ANCHOR_EMA, 0), (torch.bfloat16, tfb.TF_ANCHOR_INCL_MEAN, 0)])
+def test_decode_steps_match_oracle(dtype, mode, window):
+    """A prefill of 70 tokens seeds the anchors through tf_kv_stats' carry; then 90 decode steps run in
+    lockstep with the oracle: scores within 1e-5, thresholds within 1e-6, skip decisions equal unless the
+    score is within 1e-5 of the threshold (then the oracle's state is forced on so the runs stay comparable),
+    outputs within the attention tolerance; skipped rows are zero."""
+    B, S0, T, Hq, Hkv = 2, 70, 90, 8, 2
+    S = S0 + T
+    q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=123, dup=0.4)
+    qn, kn, vn = oracle_inputs(q, k, v)
+    ctx = tfb.Context(0)
+    params = tfb.default_params(prune_ratio=0.25, warmup_tokens=4, anchor_mode=mode, gamma=0.9)
+    st = tfb.DecodeState(B, Hkv, DEV, tau0=0.3)
+    # prefill: anchors from the first S0 tokens
+    pshape = tfb.make_shape(None, k[:, :S0], v[:, :S0])
+    ctx.ensure_workspace(pshape, params)
+    sk = torch.empty(B, S0, Hkv, device=DEV); sv = torch.empty_like(sk)
+    ctx.tf_kv_stats(pshape, params, k[:, :S0], v[:, :S0], sk, sv,
+                    tfb.tf_carry(None, None, None, st.sum_k.data_ptr(), st.sum_v.data_ptr()))
+    st.count.fill_(S0)
+    ost = oracle.decode_state(B, Hkv, 128, tau0=0.3)
+    _, sum_k = oracle.anchor_similarity(kn[:, :S0], mode, 0.9, want_sum_out=True)
+    _, sum_v = oracle.anchor_similarity(vn[:, :S0], mode, 0.9, want_sum_out=True)
+    ost["sum_k"][:] = sum_k; ost["sum_v"][:] = sum_v; ost["count"][:] = S0
+    assert np.abs(to_np(st.sum_k) - sum_k).max() < 1e-3
+
+    shape = tfb.make_shape(None, k, v, window=window, n_q_heads=Hq)
+    O = torch.full((B, Hq, 128), float("nan"), dtype=dtype, device=DEV)
+    shape.q_stride[:] = [q.stride(0), 0, q.stride(2)]
+    shape.o_stride[:] = [O.stride(0), 0, O.stride(1)]
+    score = torch.empty(B, device=DEV); skip = torch.empty(B, dtype=torch.uint8, device=DEV)
+    near, n_skips = 0, 0
+    for t in range(S0, S):
+        pos = torch.full((B,), t, dtype=torch.int32, device=DEV)
+        ctx.tf_decode_step(shape, params, 0.05, q[:, t], k, v, pos, st, O, score, skip)
+        ref = oracle.decode_step(ost, qn[:, t], kn, vn, np.full(B, t), target_ratio=0.25, eta=0.05, warmup_tokens=4,
+                                 anchor_mode=mode, gamma=0.9, window=window)
+        assert np.abs(to_np(score) - ref["score"]).max() < SCORE_ATOL
+        assert np.abs(to_np(st.tau) - ref["tau"]).max() < 1e-6
+        g_skip = skip.cpu().numpy()
+        for b in range(B):
+            if g_skip[b] != ref["skip"][b]:
+                assert abs(ref["score"][b] - ref["tau"][b]) < 1e-5, (t, b, ref["score"][b], ref["tau"][b])
+                near += 1
+        if np.array_equal(g_skip, ref["skip"]):
+            o = to_np(O)
+            assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
+            assert np.all(o[ref["skip"] == 1] == 0.0)
+        else:   # keep the two runs on the same trajectory
+            st.steps.copy_(torch.from_numpy(ost["steps"])); st.skips.copy_(torch.from_numpy(ost["skips"]))
+        n_skips += int(ref["skip"].sum())
+    code, det = ctx.tf_get_status()
+    assert code == tfb.TF_OK, det
+    assert np.array_equal(st.count.cpu().numpy(), ost["count"]) and np.array_equal(st.steps.cpu().numpy(), ost["steps"])
+    assert 0 < n_skips < B * T            # the case exercises both branches
+    assert near <= 2
+    ctx.close()

@@ -365,3 +365,60 @@ def test_tail_policy_paper_example_and_budget():
         r = orc.tail_policy(pg, y, L)
         assert abs(sum(r) / L - pg) < 1e-12
         assert all(x == 0.0 for x in r[: L - round(y * L)])
+
+
+# ------------------------------------------------------------------------------- online decode step
+def _decode_run(K, V, Q, **kw):
+    B, S, Hkv, d = K.shape
+    st = orc.decode_state(B, Hkv, d, tau0=kw.pop("tau0", 0.0))
+    out = []
+    for t in range(S):
+        out.append(orc.decode_step(st, Q[:, t], K, V, np.full(B, t), **kw))
+    return st, out
+
+
+def test_decode_steps_reproduce_the_prefill_scores_and_dense_attention():
+    """Token by token with a threshold nothing reaches: the scores are the prefill oracle's scores at every
+    position (same anchors, same order of compare and update) and the outputs are dense causal attention."""
+    rng = np.random.default_rng(5)
+    B, S, Hq, Hkv, d = 2, 40, 4, 2, 128
+    Q = rng.standard_normal((B, S, Hq, d)).astype(np.float32)
+    K = rng.standard_normal((B, S, Hkv, d)).astype(np.float32)
+    V = rng.standard_normal((B, S, Hkv, d)).astype(np.float32)
+    K[:, 20] = K[:, 3] * 1.5
+    for mode, gamma in [(orc.ANCHOR_PAST_MEAN, 0.9), (orc.ANCHOR_INCL_MEAN, 0.9), (orc.ANCHOR_EMA, 0.8)]:
+        ref = orc.layer_filter(Q, K, V, prune_ratio=0.0, window=7, anchor_mode=mode, gamma=gamma)
+        st, out = _decode_run(K, V, Q, tau0=10.0, eta=0.0, window=7, anchor_mode=mode, gamma=gamma)
+        sc = np.stack([o["score"] for o in out], 1)
+        assert np.abs(sc - ref["score"]).max() < 1e-12
+        O = np.stack([o["O"] for o in out], 1)
+        assert np.abs(O - ref["O"]).max() < 1e-10
+        assert all(o["skip"].sum() == 0 for o in out)
+        assert np.all(st["count"] == S) and np.all(st["steps"] == S) and np.all(st["skips"] == 0)
+
+
+def test_decode_threshold_feedback_signs_warmup_and_fixed_point():
+    """Section 3.3: the threshold rises while the skip ratio is above target and falls while below; with
+    Algorithm 1's printed sign it moves the other way.  Warm-up tokens are never skipped but are counted.
+    On a long stream of scores the skip ratio settles at the target."""
+    rng = np.random.default_rng(6)
+    B, S, H, d = 1, 3000, 2, 16
+    base = rng.standard_normal((1, 1, H, d))
+    K = (base + 0.8 * rng.standard_normal((B, S, H, d))).astype(np.float32)
+    V = (base + 0.8 * rng.standard_normal((B, S, H, d))).astype(np.float32)
+    Q = rng.standard_normal((B, S, H, d)).astype(np.float32)
+    st, out = _decode_run(K, V, Q, tau0=0.0, eta=0.1, target_ratio=0.3, warmup_tokens=8)
+    taus = np.array([o["tau"][0] for o in out]); skips = np.array([o["skip"][0] for o in out])
+    assert skips[:8].sum() == 0                                   # never inside the warm-up
+    assert st["skips"][0] >= skips.sum()                          # but decided skips are counted there too
+    rho = np.cumsum([1 if np.float32(o["score"][0]) > o["tau"][0] else 0 for o in out])
+    # the update uses the ratio BEFORE the current decision
+    prev_rho = np.concatenate([[0.0], rho[:-1] / np.arange(1, S)])
+    d_tau = np.diff(np.concatenate([[0.0], taus]))
+    assert np.all(np.sign(d_tau[1:]) == np.sign(np.float32(prev_rho[1:] - 0.3)))
+    assert abs(st["skips"][0] / st["steps"][0] - 0.3) < 0.03     # settles at the target
+    st2, out2 = _decode_run(K, V, Q, tau0=0.0, eta=0.1, target_ratio=0.3, warmup_tokens=8, alg1_sign=True)
+    assert out2[0]["tau"][0] > 0 > out[0]["tau"][0]               # first update: rho = 0 < target
+    # positive feedback runs away: everything or nothing is skipped in the end
+    r2 = st2["skips"][0] / st2["steps"][0]
+    assert r2 < 0.02 or r2 > 0.98
