@@ -28,7 +28,7 @@ TF_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
-           "tf_status_string", "tf_tail_policy", "tf_decode_step")
+           "tf_status_string", "tf_tail_policy", "tf_decode_step", "tf_set_scan_path")
 
 
 class tf_shape(C.Structure):
@@ -237,6 +237,10 @@ class Context:
     def tf_set_attention_path(self, path):
         """0 / False: CUDA-core kernel; 1 / True: tensor-core kernel (form chosen by size); 2: shared form; 3: split form."""
         _check(lib().tf_set_attention_path(self._h, C.c_int(int(path))), "tf_set_attention_path")
+
+    def tf_set_scan_path(self, path: int):
+        """0: choose; 1: plain CUDA-core similarity scan; 2: Gram-matrix scan on the tensor cores (bf16 sums)."""
+        _check(lib().tf_set_scan_path(self._h, C.c_int(int(path))), "tf_set_scan_path")
 
     @property
     def launches(self) -> int:

@@ -393,6 +393,12 @@ tf_status tf_set_attention_path(tf_ctx* ctx, int use_tensor_cores) {
     return TF_OK;
 }
 
+tf_status tf_set_scan_path(tf_ctx* ctx, int path) {
+    if (!ctx || path < 0 || path > 2) return TF_ERR_INVALID_ARG;
+    ctx->scan_path = path;
+    return TF_OK;
+}
+
 const char* tf_status_string(tf_status s) {
     switch (s) {
         case TF_OK: return "ok";

@@ -121,6 +121,7 @@ struct tf_ctx {
     tf::ScanScratch scan_user;     // scan bookkeeping of the caller's workspace
     tf::ScanScratch scan_owned;    // ... and of owned_ws
     int use_tensor_cores;          // bf16 attention path
+    int scan_path;                 // tf_kv_stats: 0 = choose, 1 = plain CUDA-core kernel, 2 = Gram-matrix kernel (bf16 sums)
     int attention_form;            // tensor-core kernel: 0 = choose by grid size, 1 = shared K/V tiles, 2 = split K/V tiles
     long long launches;            // kernels launched through this context
     // tf_layer_filter_host staging (owned, grown on demand)
@@ -145,6 +146,11 @@ ScanPlan scan_plan(const tf_shape& s);
 cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                             const void* K, const void* V, float* sim_k, float* sim_v,
                             const tf_carry* carry, ScanScratch* scan_scratch, cudaStream_t st);
+// bf16 running-sum anchors through 128-token Gram matrices on the tensor cores (tf_scan_tc.cu)
+bool kv_stats_gram_usable(const tf_shape& s, const tf_filter_params& p);
+cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                                 const void* K, const void* V, float* sim_k, float* sim_v,
+                                 const tf_carry* carry, ScanScratch* scan_scratch, cudaStream_t st);
 cudaError_t launch_score_fuse(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                               const float* sim_k, const float* sim_v, float* score, cudaStream_t st);
 cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,

@@ -1,0 +1,436 @@
+// Steps a1+a2 for bf16 tensors with running-sum anchors, rearranged so that the CUDA cores touch
+// O(tokens) values per tile instead of O(tokens x dims):
+//
+// For a tile X of 128 tokens of one (sequence, KV head) and the sum C of everything before it,
+//   <x_i, P_i>   = <x_i, C> + sum_{j<i} G_ij        with  G = X X^T  (128 x 128)
+//   ||x_i||^2    = G_ii
+//   ||P_{i+1}||^2 = ||P_i||^2 + 2 <x_i, P_i> + G_ii  (a prefix sum over the tile, seeded with ||C||^2)
+//   column sums of X (the tile's aggregate for the look-back) = X^T 1
+// G, X^T 1 and X C are small dense products; they run on the tensor cores (tcgen05, operands in
+// shared memory exactly as TMA delivers them, accumulators in TMEM), C entering as three bf16
+// terms c1+c2+c3 so that the fp32 carry loses nothing.  Thread i then owns token row i: it adds
+// the part of row i of G left of the diagonal, joins a block-wide prefix sum and writes the two
+// cosines.  The fp32 instruction stream per (token, head) drops from ~130 to ~20 warp
+// instructions, which is what kept the plain kernel from reaching the memory roofline.
+//
+// One CTA (128 threads) per tile, tiles by atomic ticket, carries through the same tagged records
+// and fixed-association look-back as the plain kernel (see tf_scan.cu).  TMEM: 128 columns per
+// CTA, reused in turn for X^T 1, G_K, G_V and X C.  All waits are bounded.
+#include "tf_ptx.cuh"
+
+namespace tf {
+namespace {
+
+constexpr int kGT = 128;                       // tokens per tile
+constexpr int kHalf = 128 * 128;               // one [128 rows][128 B] swizzled block
+constexpr int kXBytes = 2 * kHalf;             // one tensor's tile
+constexpr int kBtBytes = 2 * 16 * 128;         // small B operand: [16 rows][128 elements], two 64-element blocks
+constexpr int kGramAnchorEvery = 8;
+constexpr int kGramPollBatch = 4;
+constexpr uint32_t kGramTmemCols = 128;
+constexpr long long kGramWaitCycles = 1000000000ll;
+
+constexpr int kOffXk = 0, kOffXv = kXBytes, kOffBt = 2 * kXBytes, kOffMisc = kOffBt + kBtBytes;
+constexpr int kGramSmem = kOffMisc + 256 + 1024;
+
+struct GramParams {
+    int S, H, n_chains, n_chunks;
+    int incl;
+    const float* sum_k_in; const float* sum_v_in; const long long* count_in;
+    float* sum_k_out; float* sum_v_out;
+    float* sim_k; float* sim_v;
+    unsigned int* ticket; unsigned int ticket_base, epoch;
+    uint4* agg_rec; uint4* prefix_rec;
+    DevStatus* status;
+    int max_polls;
+};
+
+__device__ __forceinline__ uint4 ld_packet(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ void st_packet(uint4* p, float k, float v, unsigned int tag) {
+    asm volatile("st.volatile.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(__float_as_uint(k)), "r"(__float_as_uint(v)), "r"(tag), "r"(0u) : "memory");
+}
+__device__ __forceinline__ uint4 wait_packet(const uint4* p, uint4 first, unsigned int epoch, int max_polls,
+                                             DevStatus* status, unsigned long long where) {
+    uint4 r = first;
+    int polls = 0;
+    while (r.z != epoch) {
+        if (++polls > max_polls) {
+            report_error(status, TF_ERR_TIMEOUT, where);
+            r = make_uint4(0u, 0u, epoch, 0u);
+            break;
+        }
+        __nanosleep(32);
+        r = ld_packet(p);
+    }
+    return r;
+}
+
+// ---- tcgen05 wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptors (sm_100: version 1 at bit 46, 128-byte swizzle at 61-63); 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {   // next 64 MN elements one [128][128 B] block later
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(kHalf >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// instruction descriptors: D fp32, A/B bf16, M = 128
+constexpr uint32_t idesc(uint32_t n, bool a_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn ? (1u << 15) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+constexpr uint32_t kIdescG = idesc(128, false);    // G = X X^T
+constexpr uint32_t kIdescAgg = idesc(16, true);    // X^T Bt^T  (A = X taken MN-major: rows = dims)
+constexpr uint32_t kIdescU = idesc(16, false);     // X Bt^T
+
+// byte offset of element (row n, index k) of the small B operand (K-major, 128-byte swizzle)
+__device__ __forceinline__ uint32_t bt_off(int n, int k) {
+    return (uint32_t)((k >> 6) * (16 * 128) + n * 128 + ((((k & 63) >> 3) ^ (n & 7)) << 4) + (k & 7) * 2);
+}
+__device__ __forceinline__ unsigned short bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevStatus* status,
+                                         unsigned long long where) {
+    return mbar_wait_bounded(bar, parity, abort_flag, kGramWaitCycles, status, where);
+}
+
+__global__ void __launch_bounds__(128, 3)
+kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_tma = sbase + kOffMisc, bar_mma = bar_tma + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc + 16);
+    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(smem + kOffMisc + 20);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 24);
+    float* red = reinterpret_cast<float*>(smem + kOffMisc + 32);     // [4 warps][4] scratch for block reductions / scans
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        *s_ticket = atomicAdd(p.ticket, 1u) - p.ticket_base;
+        mbar_init(bar_tma, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    // small B operand: rows 0-2 / 3-5 will take the three bf16 terms of the K / V carry, row 6 is all ones, rest 0
+    *reinterpret_cast<uint4*>(smem + kOffBt + tid * 32) = make_uint4(0, 0, 0, 0);
+    *reinterpret_cast<uint4*>(smem + kOffBt + tid * 32 + 16) = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(6, tid)) = 0x3f80;
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kGramTmemCols);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
+
+    const unsigned int tile = *s_ticket;
+    const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
+    const int b = chain / p.H, h = chain % p.H;
+    const uint32_t xk = sbase + kOffXk, xv = sbase + kOffXv, bt = sbase + kOffBt;
+
+    if (tid == 0) {
+        mbar_expect_tx(bar_tma, 2 * kXBytes);
+        tma_load_4d(xk, &mapK, bar_tma, 0, h, c * kGT, b);
+        tma_load_4d(xk + kHalf, &mapK, bar_tma, 64, h, c * kGT, b);
+        tma_load_4d(xv, &mapV, bar_tma, 0, h, c * kGT, b);
+        tma_load_4d(xv + kHalf, &mapV, bar_tma, 64, h, c * kGT, b);
+    }
+    // look-back requests go out while the tile is in flight
+    const bool has_prev = c > 0;
+    const int a0 = has_prev ? ((c - 1) / kGramAnchorEvery) * kGramAnchorEvery : 0;
+    const uint4* prec = p.prefix_rec + ((size_t)(a0 / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid;
+    uint4 pfirst = make_uint4(0, 0, 0, 0);
+    if (has_prev) pfirst = ld_packet(prec);
+
+    uint32_t mma_phase = 0;
+    wait_bar(bar_tma, 0, abort_flag, p.status, 100);
+
+    // ---- 1. column sums: (X^T Bt^T)[d][6] = sum_t X[t][d] ---------------------------------------------
+    if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const uint32_t xa = t ? xv : xk;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)     // 16 tokens per step
+                mma_ss(tmem + 16 * t, desc_mnmajor(xa + kk * 16 * 128), desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32),
+                       kIdescAgg, kk > 0);
+        }
+        mma_commit(bar_mma);
+    }
+    wait_bar(bar_mma, mma_phase, abort_flag, p.status, 101); mma_phase ^= 1;
+    tc_fence_after();
+    float agg_k, agg_v;
+    {
+        uint32_t r0[8], r1[8];
+        tmem_ld8(tm_lane, r0);
+        tmem_ld8(tm_lane + 16, r1);
+        tmem_wait_ld();
+        agg_k = __uint_as_float(r0[6]);
+        agg_v = __uint_as_float(r1[6]);
+    }
+    if (c + 1 < p.n_chunks) st_packet(p.agg_rec + (size_t)tile * kHeadDim + tid, agg_k, agg_v, p.epoch);
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- 2. G = X X^T for K, then V; thread i adds row i left of the diagonal --------------------------
+    float r_sum[2], g_diag[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t xa = t ? xv : xk;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {   // 16 dims per step
+                const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * 32;
+                mma_ss(tmem, desc_kmajor(xa + off), desc_kmajor(xa + off), kIdescG, kk > 0);
+            }
+            mma_commit(bar_mma);
+        }
+        wait_bar(bar_mma, mma_phase, abort_flag, p.status, 102 + t); mma_phase ^= 1;
+        tc_fence_after();
+        float rs = 0.f, gd = 0.f;
+        for (int cc = 0; cc <= warp; ++cc) {          // column blocks at or left of this warp's diagonal block
+            uint32_t g[32];
+            tmem_ld32(tm_lane + cc * 32, g);
+            tmem_wait_ld();
+            if (cc < warp) {
+                float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int e = 0; e < 32; ++e) s4[e & 3] += __uint_as_float(g[e]);
+                rs += (s4[0] + s4[1]) + (s4[2] + s4[3]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float x = __uint_as_float(g[e]);
+                    rs += (e < lane) ? x : 0.f;
+                    gd = (e == lane) ? x : gd;
+                }
+            }
+        }
+        r_sum[t] = rs; g_diag[t] = gd;
+        tc_fence_before();
+        __syncthreads();
+    }
+
+    // ---- 3. carry from earlier chunks (thread = dim) -----------------------------------------------------
+    float carry_k = 0.f, carry_v = 0.f;
+    if (c == 0) {
+        if (p.sum_k_in) carry_k = p.sum_k_in[(size_t)chain * kHeadDim + tid];
+        if (p.sum_v_in) carry_v = p.sum_v_in[(size_t)chain * kHeadDim + tid];
+    } else {
+        float Ak = 0.f, Av = 0.f;
+        for (int j0 = a0; j0 < c; j0 += kGramPollBatch) {
+            uint4 r[kGramPollBatch];
+#pragma unroll
+            for (int u = 0; u < kGramPollBatch; ++u)
+                if (j0 + u < c) r[u] = ld_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
+#pragma unroll
+            for (int u = 0; u < kGramPollBatch; ++u) {
+                if (j0 + u < c) {
+                    r[u] = wait_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u],
+                                       p.epoch, p.max_polls, p.status, tile);
+                    Ak += __uint_as_float(r[u].x);
+                    Av += __uint_as_float(r[u].y);
+                }
+            }
+        }
+        pfirst = wait_packet(prec, pfirst, p.epoch, p.max_polls, p.status, tile);
+        carry_k = __uint_as_float(pfirst.x) + Ak;
+        carry_v = __uint_as_float(pfirst.y) + Av;
+    }
+    if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
+        st_packet(p.prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, p.epoch);
+    if (c + 1 == p.n_chunks) {
+        if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = carry_k + agg_k;
+        if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = carry_v + agg_v;
+    }
+
+    // ---- 4. u = X C: the carry goes into rows 0-5 of the small operand as c1 + c2 + c3 (bf16 each) --------
+    {
+        float ck = carry_k, cv = carry_v;
+#pragma unroll
+        for (int n = 0; n < 3; ++n) {
+            const unsigned short hk = bf16_bits(ck), hv = bf16_bits(cv);
+            *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(n, tid)) = hk;
+            *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(3 + n, tid)) = hv;
+            ck -= __uint_as_float((uint32_t)hk << 16);
+            cv -= __uint_as_float((uint32_t)hv << 16);
+        }
+    }
+    // ||C||^2 per tensor (block sum over dims)
+    float ck2 = warp_sum(carry_k * carry_k), cv2 = warp_sum(carry_v * carry_v);
+    if (lane == 0) { red[warp * 4 + 0] = ck2; red[warp * 4 + 1] = cv2; }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    ck2 = (red[0] + red[4]) + (red[8] + red[12]);
+    cv2 = (red[1] + red[5]) + (red[9] + red[13]);
+    if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const uint32_t xa = t ? xv : xk;
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)     // 16 dims per step
+                mma_ss(tmem + 16 * t, desc_kmajor(xa + (kk >> 2) * kHalf + (kk & 3) * 32),
+                       desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescU, kk > 0);
+        }
+        mma_commit(bar_mma);
+    }
+    wait_bar(bar_mma, mma_phase, abort_flag, p.status, 104); mma_phase ^= 1;
+    tc_fence_after();
+    float dk, dv;
+    {
+        uint32_t r0[8], r1[8];
+        tmem_ld8(tm_lane, r0);
+        tmem_ld8(tm_lane + 16, r1);
+        tmem_wait_ld();
+        dk = (__uint_as_float(r0[0]) + __uint_as_float(r0[1])) + __uint_as_float(r0[2]) + r_sum[0];   // <x_i, P_i>
+        dv = (__uint_as_float(r1[3]) + __uint_as_float(r1[4])) + __uint_as_float(r1[5]) + r_sum[1];
+    }
+
+    // ---- 5. ||P_i||^2 by a block-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosines ---------
+    float bk = fmaf(2.f, dk, g_diag[0]), bv = fmaf(2.f, dv, g_diag[1]);
+    float ik = bk, iv = bv;                                  // inclusive warp scan
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float nk = __shfl_up_sync(0xffffffffu, ik, o), nv = __shfl_up_sync(0xffffffffu, iv, o);
+        if (lane >= o) { ik += nk; iv += nv; }
+    }
+    __syncthreads();                                          // red[] is reused
+    if (lane == 31) { red[warp * 4 + 2] = ik; red[warp * 4 + 3] = iv; }
+    __syncthreads();
+    float offk = ck2, offv = cv2;
+    for (int w2 = 0; w2 < warp; ++w2) { offk += red[w2 * 4 + 2]; offv += red[w2 * 4 + 3]; }
+    float ppk = offk + (ik - bk), ppv = offv + (iv - bv);    // ||P_i||^2 (exclusive)
+    const int t_tok = c * kGT + tid;
+    if (t_tok < p.S) {
+        if (p.incl) { dk += g_diag[0]; dv += g_diag[1]; ppk += bk; ppv += bv; }
+        const long long cnt = (p.count_in ? p.count_in[b] : 0ll) + t_tok + (p.incl ? 1 : 0);
+        float cosk = 0.f, cosv = 0.f;
+        if (cnt > 0) {
+            const float s = 1.f / (float)cnt;               // anchor = sum * s
+            cosk = (dk * s) / (fmaxf(sqrtf(g_diag[0]), kNormEps) * fmaxf(sqrtf(fmaxf(ppk, 0.f)) * s, kNormEps));
+            cosv = (dv * s) / (fmaxf(sqrtf(g_diag[1]), kNormEps) * fmaxf(sqrtf(fmaxf(ppv, 0.f)) * s, kNormEps));
+        }
+        const size_t o = ((size_t)b * p.S + t_tok) * p.H + h;
+        p.sim_k[o] = cosk;
+        p.sim_v[o] = cosv;
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) { }
+        __syncthreads();
+    }
+    if (warp == 0) tmem_dealloc(tmem, kGramTmemCols);
+}
+
+}  // namespace
+
+bool kv_stats_gram_usable(const tf_shape& s, const tf_filter_params& p) {
+    return s.dtype == TF_BF16 && p.anchor_mode != TF_ANCHOR_EMA;
+}
+
+cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
+                                 const void* K, const void* V, float* sim_k, float* sim_v,
+                                 const tf_carry* carry, ScanScratch* ws, cudaStream_t st) {
+    const int n_chains = s.batch * s.n_kv_heads;
+    const int n_chunks = (s.seq + kGT - 1) / kGT;
+    const size_t tiles = (size_t)n_chains * (size_t)n_chunks;
+    if (tiles == 0) return cudaSuccess;
+    if (tiles > 0x7fffffffu) return cudaErrorInvalidValue;
+    const size_t anchors = (size_t)n_chains * (size_t)((n_chunks + kGramAnchorEvery - 1) / kGramAnchorEvery);
+    const size_t agg_offset = 256, prefix_offset = agg_offset + tiles * kHeadDim * sizeof(uint4);
+    // (a tag distinguishes this kernel's record layout from the plain kernel's, which may share the scratch)
+    const size_t bytes = ((prefix_offset + anchors * kHeadDim * sizeof(uint4) + 255) / 256 * 256) | 1;
+    if (ws->needs_clear || ws->bytes != bytes || ws->epoch == 0xffffffffu) {
+        cudaError_t e = cudaMemsetAsync(ws->ptr, 0, bytes & ~(size_t)1, st);
+        if (e != cudaSuccess) return e;
+        ws->needs_clear = false;
+        ws->bytes = bytes;
+        ws->epoch = 0;
+        ws->ticket_base = 0;
+    }
+    ws->epoch += 1;
+
+    CUtensorMap mk, mv;
+    if (!make_bshd_map(&mk, K, s.k_stride, s.batch, s.seq, s.n_kv_heads, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kGT,
+                       CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_bshd_map(&mv, V, s.v_stride, s.batch, s.seq, s.n_kv_heads, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kGT,
+                       CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorNotSupported;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kv_stats_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGramSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    GramParams gp{};
+    gp.S = s.seq; gp.H = s.n_kv_heads; gp.n_chains = n_chains; gp.n_chunks = n_chunks;
+    gp.incl = (p.anchor_mode == TF_ANCHOR_INCL_MEAN);
+    if (carry) {
+        gp.sum_k_in = carry->sum_k_in; gp.sum_v_in = carry->sum_v_in;
+        gp.count_in = reinterpret_cast<const long long*>(carry->count_in);
+        gp.sum_k_out = carry->sum_k_out; gp.sum_v_out = carry->sum_v_out;
+    }
+    gp.sim_k = sim_k; gp.sim_v = sim_v;
+    char* base = static_cast<char*>(ws->ptr);
+    gp.ticket = reinterpret_cast<unsigned int*>(base);
+    gp.ticket_base = ws->ticket_base;
+    gp.epoch = ws->epoch;
+    gp.agg_rec = reinterpret_cast<uint4*>(base + agg_offset);
+    gp.prefix_rec = reinterpret_cast<uint4*>(base + prefix_offset);
+    gp.status = ctx->dev_status;
+    gp.max_polls = 1 << 20;
+    ws->ticket_base += (unsigned int)tiles;
+    kv_stats_gram_kernel<<<(unsigned)tiles, 128, kGramSmem, st>>>(gp, mk, mv);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace tf
