@@ -139,13 +139,11 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar_tma = sbase + kOffMisc, bar_mma = bar_tma + 8;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc + 16);
-    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(smem + kOffMisc + 20);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 24);
     float* red = reinterpret_cast<float*>(smem + kOffMisc + 32);     // [4 warps][4] scratch for block reductions / scans
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        *s_ticket = atomicAdd(p.ticket, 1u) - p.ticket_base;
         mbar_init(bar_tma, 1);
         mbar_init(bar_mma, 1);
         *abort_flag = 0;
@@ -156,7 +154,7 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
     *reinterpret_cast<uint4*>(smem + kOffBt + tid * 32 + 16) = make_uint4(0, 0, 0, 0);
     __syncthreads();
     *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(6, tid)) = 0x3f80;
-    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kGramTmemCols);
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kGramTmemCols);
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -164,7 +162,10 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
     const uint32_t tmem = *tmem_slot;
     const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
 
-    const unsigned int tile = *s_ticket;
+    // Tiles go by block index.  CTAs are started in index order, so the records a tile waits for belong to
+    // tiles that were started before it; should a scheduler ever break that order, the bounded waits turn the
+    // stall into TF_ERR_TIMEOUT instead of a hang.
+    const unsigned int tile = blockIdx.x;
     const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
     const int b = chain / p.H, h = chain % p.H;
     const uint32_t xk = sbase + kOffXk, xv = sbase + kOffXv, bt = sbase + kOffBt;
@@ -189,30 +190,69 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
     // ---- 1. column sums: (X^T Bt^T)[d][6] = sum_t X[t][d] ---------------------------------------------
     if (tid == 0) {
         tc_fence_after();
+        // a 16-column product depends on the one before it through its accumulator: four independent
+        // chains (tensor x parity of the step) are interleaved and added up after the read
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const uint32_t xa = t ? xv : xk;
+        for (int kk = 0; kk < 8; ++kk)         // 16 tokens per step
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)     // 16 tokens per step
-                mma_ss(tmem + 16 * t, desc_mnmajor(xa + kk * 16 * 128), desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32),
-                       kIdescAgg, kk > 0);
-        }
+            for (int t = 0; t < 2; ++t)
+                mma_ss(tmem + 32 * t + 16 * (kk & 1), desc_mnmajor((t ? xv : xk) + kk * 16 * 128),
+                       desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescAgg, kk > 1);
         mma_commit(bar_mma);
     }
     wait_bar(bar_mma, mma_phase, abort_flag, p.status, 101); mma_phase ^= 1;
     tc_fence_after();
     float agg_k, agg_v;
     {
-        uint32_t r0[8], r1[8];
-        tmem_ld8(tm_lane, r0);
-        tmem_ld8(tm_lane + 16, r1);
+        uint32_t r0[8], r1[8], r2[8], r3[8];
+        tmem_ld8(tm_lane, r0); tmem_ld8(tm_lane + 16, r1);
+        tmem_ld8(tm_lane + 32, r2); tmem_ld8(tm_lane + 48, r3);
         tmem_wait_ld();
-        agg_k = __uint_as_float(r0[6]);
-        agg_v = __uint_as_float(r1[6]);
+        agg_k = __uint_as_float(r0[6]) + __uint_as_float(r1[6]);
+        agg_v = __uint_as_float(r2[6]) + __uint_as_float(r3[6]);
     }
     if (c + 1 < p.n_chunks) st_packet(p.agg_rec + (size_t)tile * kHeadDim + tid, agg_k, agg_v, p.epoch);
     tc_fence_before();
     __syncthreads();
+
+    // ---- carry from earlier chunks (thread = dim).  A tile that publishes a prefix (every 8th chunk) does this
+    // before its Gram matrices: its prefix depends on older tiles only, and the seven tiles after it wait for it.
+    float carry_k = 0.f, carry_v = 0.f;
+    auto resolve_carry = [&]() {
+    if (c == 0) {
+        if (p.sum_k_in) carry_k = p.sum_k_in[(size_t)chain * kHeadDim + tid];
+        if (p.sum_v_in) carry_v = p.sum_v_in[(size_t)chain * kHeadDim + tid];
+    } else {
+        float Ak = 0.f, Av = 0.f;
+        for (int j0 = a0; j0 < c; j0 += kGramPollBatch) {
+            uint4 r[kGramPollBatch];
+#pragma unroll
+            for (int u = 0; u < kGramPollBatch; ++u)
+                if (j0 + u < c) r[u] = ld_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
+#pragma unroll
+            for (int u = 0; u < kGramPollBatch; ++u) {
+                if (j0 + u < c) {
+                    r[u] = wait_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u],
+                                       p.epoch, p.max_polls, p.status, tile);
+                    Ak += __uint_as_float(r[u].x);
+                    Av += __uint_as_float(r[u].y);
+                }
+            }
+        }
+        pfirst = wait_packet(prec, pfirst, p.epoch, p.max_polls, p.status, tile);
+        carry_k = __uint_as_float(pfirst.x) + Ak;
+        carry_v = __uint_as_float(pfirst.y) + Av;
+    }
+    if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
+        st_packet(p.prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, p.epoch);
+    if (c + 1 == p.n_chunks) {
+        if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = carry_k + agg_k;
+        if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = carry_v + agg_v;
+    }
+
+    };
+    const bool publishes_prefix = (c % kGramAnchorEvery == 0);
+    if (publishes_prefix) resolve_carry();
 
     // ---- 2. G = X X^T for K, then V; thread i adds row i left of the diagonal --------------------------
     float r_sum[2], g_diag[2];
@@ -254,38 +294,7 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
         __syncthreads();
     }
 
-    // ---- 3. carry from earlier chunks (thread = dim) -----------------------------------------------------
-    float carry_k = 0.f, carry_v = 0.f;
-    if (c == 0) {
-        if (p.sum_k_in) carry_k = p.sum_k_in[(size_t)chain * kHeadDim + tid];
-        if (p.sum_v_in) carry_v = p.sum_v_in[(size_t)chain * kHeadDim + tid];
-    } else {
-        float Ak = 0.f, Av = 0.f;
-        for (int j0 = a0; j0 < c; j0 += kGramPollBatch) {
-            uint4 r[kGramPollBatch];
-#pragma unroll
-            for (int u = 0; u < kGramPollBatch; ++u)
-                if (j0 + u < c) r[u] = ld_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
-#pragma unroll
-            for (int u = 0; u < kGramPollBatch; ++u) {
-                if (j0 + u < c) {
-                    r[u] = wait_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u],
-                                       p.epoch, p.max_polls, p.status, tile);
-                    Ak += __uint_as_float(r[u].x);
-                    Av += __uint_as_float(r[u].y);
-                }
-            }
-        }
-        pfirst = wait_packet(prec, pfirst, p.epoch, p.max_polls, p.status, tile);
-        carry_k = __uint_as_float(pfirst.x) + Ak;
-        carry_v = __uint_as_float(pfirst.y) + Av;
-    }
-    if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
-        st_packet(p.prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, p.epoch);
-    if (c + 1 == p.n_chunks) {
-        if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = carry_k + agg_k;
-        if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = carry_v + agg_v;
-    }
+    if (!publishes_prefix) resolve_carry();
 
     // ---- 4. u = X C: the carry goes into rows 0-5 of the small operand as c1 + c2 + c3 (bf16 each) --------
     {
@@ -310,25 +319,24 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
     if (tid == 0) {
         tc_fence_after();
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const uint32_t xa = t ? xv : xk;
+        for (int kk = 0; kk < 8; ++kk)         // 16 dims per step; four interleaved accumulator chains as above
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)     // 16 dims per step
-                mma_ss(tmem + 16 * t, desc_kmajor(xa + (kk >> 2) * kHalf + (kk & 3) * 32),
-                       desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescU, kk > 0);
-        }
+            for (int t = 0; t < 2; ++t)
+                mma_ss(tmem + 32 * t + 16 * (kk & 1), desc_kmajor((t ? xv : xk) + (kk >> 2) * kHalf + (kk & 3) * 32),
+                       desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescU, kk > 1);
         mma_commit(bar_mma);
     }
     wait_bar(bar_mma, mma_phase, abort_flag, p.status, 104); mma_phase ^= 1;
     tc_fence_after();
     float dk, dv;
     {
-        uint32_t r0[8], r1[8];
-        tmem_ld8(tm_lane, r0);
-        tmem_ld8(tm_lane + 16, r1);
+        uint32_t r0[8], r1[8], r2[8], r3[8];
+        tmem_ld8(tm_lane, r0); tmem_ld8(tm_lane + 16, r1);
+        tmem_ld8(tm_lane + 32, r2); tmem_ld8(tm_lane + 48, r3);
         tmem_wait_ld();
-        dk = (__uint_as_float(r0[0]) + __uint_as_float(r0[1])) + __uint_as_float(r0[2]) + r_sum[0];   // <x_i, P_i>
-        dv = (__uint_as_float(r1[3]) + __uint_as_float(r1[4])) + __uint_as_float(r1[5]) + r_sum[1];
+        auto f = [](uint32_t a, uint32_t b2) { return __uint_as_float(a) + __uint_as_float(b2); };
+        dk = (f(r0[0], r1[0]) + f(r0[1], r1[1])) + f(r0[2], r1[2]) + r_sum[0];   // <x_i, P_i>
+        dv = (f(r2[3], r3[3]) + f(r2[4], r3[4])) + f(r2[5], r3[5]) + r_sum[1];
     }
 
     // ---- 5. ||P_i||^2 by a block-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosines ---------
@@ -367,7 +375,7 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
         while (clock64() - t0 < 2000000ll) { }
         __syncthreads();
     }
-    if (warp == 0) tmem_dealloc(tmem, kGramTmemCols);
+    if (warp == 1) tmem_dealloc(tmem, kGramTmemCols);
 }
 
 }  // namespace
