@@ -13,9 +13,11 @@
 // cosines.  The fp32 instruction stream per (token, head) drops from ~130 to ~20 warp
 // instructions, which is what kept the plain kernel from reaching the memory roofline.
 //
-// One CTA (128 threads) per tile, tiles by atomic ticket, carries through the same tagged records
-// and fixed-association look-back as the plain kernel (see tf_scan.cu).  TMEM: 128 columns per
-// CTA, reused in turn for X^T 1, G_K, G_V and X C.  All waits are bounded.
+// One CTA (128 threads) per (tile, tensor): K and V are independent here, and the smaller footprint
+// (32 KiB of rows, 64 TMEM columns, reused in turn for X^T 1, the two halves of G and X C) lets six CTAs
+// share an SM, so that the loads of some overlap the arithmetic of others.  Carries travel through tagged
+// records with the same fixed-association look-back as the plain kernel (see tf_scan.cu); a record is 128
+// 8-byte packets {value, tag}.  All waits are bounded.
 #include "tf_ptx.cuh"
 
 namespace tf {
@@ -27,49 +29,7 @@ constexpr int kXBytes = 2 * kHalf;             // one tensor's tile
 constexpr int kBtBytes = 2 * 16 * 128;         // small B operand: [16 rows][128 elements], two 64-element blocks
 constexpr int kGramAnchorEvery = 8;
 constexpr int kGramPollBatch = 4;
-constexpr uint32_t kGramTmemCols = 128;
 constexpr long long kGramWaitCycles = 1000000000ll;
-
-constexpr int kOffXk = 0, kOffXv = kXBytes, kOffBt = 2 * kXBytes, kOffMisc = kOffBt + kBtBytes;
-constexpr int kGramSmem = kOffMisc + 256 + 1024;
-
-struct GramParams {
-    int S, H, n_chains, n_chunks;
-    int incl;
-    const float* sum_k_in; const float* sum_v_in; const long long* count_in;
-    float* sum_k_out; float* sum_v_out;
-    float* sim_k; float* sim_v;
-    unsigned int* ticket; unsigned int ticket_base, epoch;
-    uint4* agg_rec; uint4* prefix_rec;
-    DevStatus* status;
-    int max_polls;
-};
-
-__device__ __forceinline__ uint4 ld_packet(const uint4* p) {
-    uint4 r;
-    asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
-    return r;
-}
-__device__ __forceinline__ void st_packet(uint4* p, float k, float v, unsigned int tag) {
-    asm volatile("st.volatile.global.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(__float_as_uint(k)), "r"(__float_as_uint(v)), "r"(tag), "r"(0u) : "memory");
-}
-__device__ __forceinline__ uint4 wait_packet(const uint4* p, uint4 first, unsigned int epoch, int max_polls,
-                                             DevStatus* status, unsigned long long where) {
-    uint4 r = first;
-    int polls = 0;
-    while (r.z != epoch) {
-        if (++polls > max_polls) {
-            report_error(status, TF_ERR_TIMEOUT, where);
-            r = make_uint4(0u, 0u, epoch, 0u);
-            break;
-        }
-        __nanosleep(32);
-        r = ld_packet(p);
-    }
-    return r;
-}
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -117,7 +77,6 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {   // next 64 M
 constexpr uint32_t idesc(uint32_t n, bool a_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn ? (1u << 15) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
-constexpr uint32_t kIdescG = idesc(128, false);    // G = X X^T
 constexpr uint32_t kIdescAgg = idesc(16, true);    // X^T Bt^T  (A = X taken MN-major: rows = dims)
 constexpr uint32_t kIdescU = idesc(16, false);     // X Bt^T
 
@@ -132,15 +91,62 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return mbar_wait_bounded(bar, parity, abort_flag, kGramWaitCycles, status, where);
 }
 
-__global__ void __launch_bounds__(128, 3)
-kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+// ---- 8-byte record packets {value, tag}: one tensor per CTA --------------------------------------------
+__device__ __forceinline__ uint2 ld_packet2(const uint2* p) {
+    uint2 r;
+    asm volatile("ld.volatile.global.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ void st_packet2(uint2* p, float v, unsigned int tag) {
+    asm volatile("st.volatile.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(__float_as_uint(v)), "r"(tag) : "memory");
+}
+__device__ __forceinline__ float wait_packet2(const uint2* p, uint2 first, unsigned int epoch, int max_polls,
+                                              DevStatus* status, unsigned long long where) {
+    uint2 r = first;
+    int polls = 0;
+    while (r.y != epoch) {
+        if (++polls > max_polls) {
+            report_error(status, TF_ERR_TIMEOUT, where);
+            r.x = 0u;
+            break;
+        }
+        __nanosleep(32);
+        r = ld_packet2(p);
+    }
+    return __uint_as_float(r.x);
+}
+
+// One CTA per (tile, tensor): 32 KiB of rows, 64 TMEM columns, so six CTAs share an SM and their loads
+// overlap one another's arithmetic.
+constexpr int kT1OffX = 0, kT1OffBt = kXBytes, kT1OffMisc = kT1OffBt + kBtBytes;
+constexpr int kT1Smem = kT1OffMisc + 256;          // the dynamic segment must start 1024-byte aligned (checked)
+constexpr uint32_t kT1TmemCols = 64;
+constexpr uint32_t kIdescG64 = idesc(64, false);   // 64 columns of G at a time
+
+struct Gram1Params {
+    int S, H, n_chains, n_chunks;
+    int incl;
+    const float* sum_in[2]; const long long* count_in;
+    float* sum_out[2];
+    float* sim[2];
+    unsigned int epoch;
+    uint2* agg_rec[2]; uint2* prefix_rec[2];
+    DevStatus* status;
+    int max_polls;
+};
+
+__global__ void __launch_bounds__(128, 6)
+kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
+    extern __shared__ uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar_tma = sbase + kOffMisc, bar_mma = bar_tma + 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc + 16);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 24);
-    float* red = reinterpret_cast<float*>(smem + kOffMisc + 32);     // [4 warps][4] scratch for block reductions / scans
+    if (sbase & 1023u) {   // the swizzled operand layout needs it; nothing has been started yet
+        if (threadIdx.x == 0) report_error(p.status, TF_ERR_TIMEOUT, 199);
+        return;
+    }
+    const uint32_t bar_tma = sbase + kT1OffMisc, bar_mma = bar_tma + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kT1OffMisc + 16);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kT1OffMisc + 24);
+    float* red = reinterpret_cast<float*>(smem + kT1OffMisc + 32);     // [4 warps][2] block reduction / scan scratch
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -149,12 +155,12 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
         *abort_flag = 0;
         mbar_fence_init();
     }
-    // small B operand: rows 0-2 / 3-5 will take the three bf16 terms of the K / V carry, row 6 is all ones, rest 0
-    *reinterpret_cast<uint4*>(smem + kOffBt + tid * 32) = make_uint4(0, 0, 0, 0);
-    *reinterpret_cast<uint4*>(smem + kOffBt + tid * 32 + 16) = make_uint4(0, 0, 0, 0);
+    // small B operand: rows 0-2 will take the three bf16 terms of the carry, row 6 is all ones, the rest 0
+    *reinterpret_cast<uint4*>(smem + kT1OffBt + tid * 32) = make_uint4(0, 0, 0, 0);
+    *reinterpret_cast<uint4*>(smem + kT1OffBt + tid * 32 + 16) = make_uint4(0, 0, 0, 0);
     __syncthreads();
-    *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(6, tid)) = 0x3f80;
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kGramTmemCols);
+    *reinterpret_cast<unsigned short*>(smem + kT1OffBt + bt_off(6, tid)) = 0x3f80;
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kT1TmemCols);
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -162,210 +168,184 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
     const uint32_t tmem = *tmem_slot;
     const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
 
-    // Tiles go by block index.  CTAs are started in index order, so the records a tile waits for belong to
-    // tiles that were started before it; should a scheduler ever break that order, the bounded waits turn the
-    // stall into TF_ERR_TIMEOUT instead of a hang.
-    const unsigned int tile = blockIdx.x;
+    // Tiles go by block index (K and V of a tile side by side).  CTAs are started in index order, so the
+    // records a tile waits for belong to tiles started before it; should a scheduler ever break that order,
+    // the bounded waits turn the stall into TF_ERR_TIMEOUT instead of a hang.
+    const int x = blockIdx.x & 1;
+    const unsigned int tile = blockIdx.x >> 1;
     const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
     const int b = chain / p.H, h = chain % p.H;
-    const uint32_t xk = sbase + kOffXk, xv = sbase + kOffXv, bt = sbase + kOffBt;
+    const uint32_t xa = sbase + kT1OffX, bt = sbase + kT1OffBt;
+    uint2* agg_rec = p.agg_rec[x];
+    uint2* prefix_rec = p.prefix_rec[x];
 
     if (tid == 0) {
-        mbar_expect_tx(bar_tma, 2 * kXBytes);
-        tma_load_4d(xk, &mapK, bar_tma, 0, h, c * kGT, b);
-        tma_load_4d(xk + kHalf, &mapK, bar_tma, 64, h, c * kGT, b);
-        tma_load_4d(xv, &mapV, bar_tma, 0, h, c * kGT, b);
-        tma_load_4d(xv + kHalf, &mapV, bar_tma, 64, h, c * kGT, b);
+        const CUtensorMap* map = x ? &mapV : &mapK;
+        mbar_expect_tx(bar_tma, kXBytes);
+        tma_load_4d(xa, map, bar_tma, 0, h, c * kGT, b);
+        tma_load_4d(xa + kHalf, map, bar_tma, 64, h, c * kGT, b);
     }
     // look-back requests go out while the tile is in flight
     const bool has_prev = c > 0;
     const int a0 = has_prev ? ((c - 1) / kGramAnchorEvery) * kGramAnchorEvery : 0;
-    const uint4* prec = p.prefix_rec + ((size_t)(a0 / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid;
-    uint4 pfirst = make_uint4(0, 0, 0, 0);
-    if (has_prev) pfirst = ld_packet(prec);
+    const uint2* prec = prefix_rec + ((size_t)(a0 / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid;
+    uint2 pfirst = make_uint2(0, 0);
+    if (has_prev) pfirst = ld_packet2(prec);
 
     uint32_t mma_phase = 0;
     wait_bar(bar_tma, 0, abort_flag, p.status, 100);
 
-    // ---- 1. column sums: (X^T Bt^T)[d][6] = sum_t X[t][d] ---------------------------------------------
+    // ---- 1. column sums: (X^T Bt^T)[d][6] = sum_t X[t][d]; two interleaved accumulator chains ------------
     if (tid == 0) {
         tc_fence_after();
-        // a 16-column product depends on the one before it through its accumulator: four independent
-        // chains (tensor x parity of the step) are interleaved and added up after the read
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)         // 16 tokens per step
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
-                mma_ss(tmem + 32 * t + 16 * (kk & 1), desc_mnmajor((t ? xv : xk) + kk * 16 * 128),
-                       desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescAgg, kk > 1);
+            mma_ss(tmem + 16 * (kk & 1), desc_mnmajor(xa + kk * 16 * 128),
+                   desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescAgg, kk > 1);
         mma_commit(bar_mma);
     }
     wait_bar(bar_mma, mma_phase, abort_flag, p.status, 101); mma_phase ^= 1;
     tc_fence_after();
-    float agg_k, agg_v;
+    float agg;
     {
-        uint32_t r0[8], r1[8], r2[8], r3[8];
-        tmem_ld8(tm_lane, r0); tmem_ld8(tm_lane + 16, r1);
-        tmem_ld8(tm_lane + 32, r2); tmem_ld8(tm_lane + 48, r3);
+        uint32_t r0[8], r1[8];
+        tmem_ld8(tm_lane, r0);
+        tmem_ld8(tm_lane + 16, r1);
         tmem_wait_ld();
-        agg_k = __uint_as_float(r0[6]) + __uint_as_float(r1[6]);
-        agg_v = __uint_as_float(r2[6]) + __uint_as_float(r3[6]);
+        agg = __uint_as_float(r0[6]) + __uint_as_float(r1[6]);
     }
-    if (c + 1 < p.n_chunks) st_packet(p.agg_rec + (size_t)tile * kHeadDim + tid, agg_k, agg_v, p.epoch);
+    if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, p.epoch);
     tc_fence_before();
     __syncthreads();
 
     // ---- carry from earlier chunks (thread = dim).  A tile that publishes a prefix (every 8th chunk) does this
-    // before its Gram matrices: its prefix depends on older tiles only, and the seven tiles after it wait for it.
-    float carry_k = 0.f, carry_v = 0.f;
+    // before its Gram matrix: its prefix depends on older tiles only, and the seven tiles after it wait for it.
+    float carry = 0.f;
     auto resolve_carry = [&]() {
-    if (c == 0) {
-        if (p.sum_k_in) carry_k = p.sum_k_in[(size_t)chain * kHeadDim + tid];
-        if (p.sum_v_in) carry_v = p.sum_v_in[(size_t)chain * kHeadDim + tid];
-    } else {
-        float Ak = 0.f, Av = 0.f;
-        for (int j0 = a0; j0 < c; j0 += kGramPollBatch) {
-            uint4 r[kGramPollBatch];
+        if (c == 0) {
+            if (p.sum_in[x]) carry = p.sum_in[x][(size_t)chain * kHeadDim + tid];
+        } else {
+            float A = 0.f;
+            for (int j0 = a0; j0 < c; j0 += kGramPollBatch) {
+                uint2 r[kGramPollBatch];
 #pragma unroll
-            for (int u = 0; u < kGramPollBatch; ++u)
-                if (j0 + u < c) r[u] = ld_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
+                for (int u = 0; u < kGramPollBatch; ++u)
+                    if (j0 + u < c) r[u] = ld_packet2(agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
 #pragma unroll
-            for (int u = 0; u < kGramPollBatch; ++u) {
-                if (j0 + u < c) {
-                    r[u] = wait_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u],
-                                       p.epoch, p.max_polls, p.status, tile);
-                    Ak += __uint_as_float(r[u].x);
-                    Av += __uint_as_float(r[u].y);
-                }
+                for (int u = 0; u < kGramPollBatch; ++u)
+                    if (j0 + u < c)
+                        A += wait_packet2(agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u], p.epoch,
+                                          p.max_polls, p.status, tile);
             }
+            carry = wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile) + A;
         }
-        pfirst = wait_packet(prec, pfirst, p.epoch, p.max_polls, p.status, tile);
-        carry_k = __uint_as_float(pfirst.x) + Ak;
-        carry_v = __uint_as_float(pfirst.y) + Av;
-    }
-    if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
-        st_packet(p.prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, p.epoch);
-    if (c + 1 == p.n_chunks) {
-        if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = carry_k + agg_k;
-        if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = carry_v + agg_v;
-    }
-
+        if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
+            st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, p.epoch);
+        if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = carry + agg;
     };
     const bool publishes_prefix = (c % kGramAnchorEvery == 0);
     if (publishes_prefix) resolve_carry();
 
-    // ---- 2. G = X X^T for K, then V; thread i adds row i left of the diagonal --------------------------
-    float r_sum[2], g_diag[2];
+    // ---- 2. G = X X^T, 64 columns at a time; thread i adds row i left of the diagonal ---------------------
+    float r_sum = 0.f, g_diag = 0.f;
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
+    for (int hh = 0; hh < 2; ++hh) {
         if (tid == 0) {
             tc_fence_after();
-            const uint32_t xa = t ? xv : xk;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {   // 16 dims per step
+            for (int kk = 0; kk < 8; ++kk) {   // 16 dims per step; B = rows 64 hh .. 64 hh + 63 of the same tile
                 const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * 32;
-                mma_ss(tmem, desc_kmajor(xa + off), desc_kmajor(xa + off), kIdescG, kk > 0);
+                mma_ss(tmem, desc_kmajor(xa + off), desc_kmajor(xa + hh * (64 * 128) + off), kIdescG64, kk > 0);
             }
             mma_commit(bar_mma);
         }
-        wait_bar(bar_mma, mma_phase, abort_flag, p.status, 102 + t); mma_phase ^= 1;
+        wait_bar(bar_mma, mma_phase, abort_flag, p.status, 102 + hh); mma_phase ^= 1;
         tc_fence_after();
-        float rs = 0.f, gd = 0.f;
-        for (int cc = 0; cc <= warp; ++cc) {          // column blocks at or left of this warp's diagonal block
+#pragma unroll
+        for (int lc = 0; lc < 2; ++lc) {
+            const int cb = 2 * hh + lc;               // 32-column block of G (warp-uniform comparisons)
+            if (cb > warp) continue;
             uint32_t g[32];
-            tmem_ld32(tm_lane + cc * 32, g);
+            tmem_ld32(tm_lane + lc * 32, g);
             tmem_wait_ld();
-            if (cc < warp) {
+            if (cb < warp) {
                 float s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int e = 0; e < 32; ++e) s4[e & 3] += __uint_as_float(g[e]);
-                rs += (s4[0] + s4[1]) + (s4[2] + s4[3]);
+                r_sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
             } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const float x = __uint_as_float(g[e]);
-                    rs += (e < lane) ? x : 0.f;
-                    gd = (e == lane) ? x : gd;
+                    const float v = __uint_as_float(g[e]);
+                    r_sum += (e < lane) ? v : 0.f;
+                    g_diag = (e == lane) ? v : g_diag;
                 }
             }
         }
-        r_sum[t] = rs; g_diag[t] = gd;
         tc_fence_before();
         __syncthreads();
     }
-
     if (!publishes_prefix) resolve_carry();
 
-    // ---- 4. u = X C: the carry goes into rows 0-5 of the small operand as c1 + c2 + c3 (bf16 each) --------
+    // ---- 3. u = X C: the carry goes into rows 0-2 of the small operand as c1 + c2 + c3 (bf16 each) ---------
     {
-        float ck = carry_k, cv = carry_v;
+        float cr = carry;
 #pragma unroll
         for (int n = 0; n < 3; ++n) {
-            const unsigned short hk = bf16_bits(ck), hv = bf16_bits(cv);
-            *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(n, tid)) = hk;
-            *reinterpret_cast<unsigned short*>(smem + kOffBt + bt_off(3 + n, tid)) = hv;
-            ck -= __uint_as_float((uint32_t)hk << 16);
-            cv -= __uint_as_float((uint32_t)hv << 16);
+            const unsigned short hb = bf16_bits(cr);
+            *reinterpret_cast<unsigned short*>(smem + kT1OffBt + bt_off(n, tid)) = hb;
+            cr -= __uint_as_float((uint32_t)hb << 16);
         }
     }
-    // ||C||^2 per tensor (block sum over dims)
-    float ck2 = warp_sum(carry_k * carry_k), cv2 = warp_sum(carry_v * carry_v);
-    if (lane == 0) { red[warp * 4 + 0] = ck2; red[warp * 4 + 1] = cv2; }
+    float c2 = warp_sum(carry * carry);            // ||C||^2 (block sum over dims)
+    if (lane == 0) red[warp * 2] = c2;
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    ck2 = (red[0] + red[4]) + (red[8] + red[12]);
-    cv2 = (red[1] + red[5]) + (red[9] + red[13]);
+    c2 = (red[0] + red[2]) + (red[4] + red[6]);
     if (tid == 0) {
         tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)         // 16 dims per step; four interleaved accumulator chains as above
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
-                mma_ss(tmem + 32 * t + 16 * (kk & 1), desc_kmajor((t ? xv : xk) + (kk >> 2) * kHalf + (kk & 3) * 32),
-                       desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescU, kk > 1);
+        for (int kk = 0; kk < 8; ++kk)             // 16 dims per step; two interleaved accumulator chains
+            mma_ss(tmem + 16 * (kk & 1), desc_kmajor(xa + (kk >> 2) * kHalf + (kk & 3) * 32),
+                   desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescU, kk > 1);
         mma_commit(bar_mma);
     }
     wait_bar(bar_mma, mma_phase, abort_flag, p.status, 104); mma_phase ^= 1;
     tc_fence_after();
-    float dk, dv;
+    float d;
     {
-        uint32_t r0[8], r1[8], r2[8], r3[8];
-        tmem_ld8(tm_lane, r0); tmem_ld8(tm_lane + 16, r1);
-        tmem_ld8(tm_lane + 32, r2); tmem_ld8(tm_lane + 48, r3);
+        uint32_t r0[8], r1[8];
+        tmem_ld8(tm_lane, r0);
+        tmem_ld8(tm_lane + 16, r1);
         tmem_wait_ld();
         auto f = [](uint32_t a, uint32_t b2) { return __uint_as_float(a) + __uint_as_float(b2); };
-        dk = (f(r0[0], r1[0]) + f(r0[1], r1[1])) + f(r0[2], r1[2]) + r_sum[0];   // <x_i, P_i>
-        dv = (f(r2[3], r3[3]) + f(r2[4], r3[4])) + f(r2[5], r3[5]) + r_sum[1];
+        d = (f(r0[0], r1[0]) + f(r0[1], r1[1])) + f(r0[2], r1[2]) + r_sum;   // <x_i, P_i>
     }
 
-    // ---- 5. ||P_i||^2 by a block-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosines ---------
-    float bk = fmaf(2.f, dk, g_diag[0]), bv = fmaf(2.f, dv, g_diag[1]);
-    float ik = bk, iv = bv;                                  // inclusive warp scan
+    // ---- 4. ||P_i||^2 by a block-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosine ----------
+    const float bi = fmaf(2.f, d, g_diag);
+    float incl_sum = bi;                           // inclusive warp scan
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const float nk = __shfl_up_sync(0xffffffffu, ik, o), nv = __shfl_up_sync(0xffffffffu, iv, o);
-        if (lane >= o) { ik += nk; iv += nv; }
+        const float n = __shfl_up_sync(0xffffffffu, incl_sum, o);
+        if (lane >= o) incl_sum += n;
     }
-    __syncthreads();                                          // red[] is reused
-    if (lane == 31) { red[warp * 4 + 2] = ik; red[warp * 4 + 3] = iv; }
+    if (lane == 31) red[warp * 2 + 1] = incl_sum;
     __syncthreads();
-    float offk = ck2, offv = cv2;
-    for (int w2 = 0; w2 < warp; ++w2) { offk += red[w2 * 4 + 2]; offv += red[w2 * 4 + 3]; }
-    float ppk = offk + (ik - bk), ppv = offv + (iv - bv);    // ||P_i||^2 (exclusive)
+    float off = c2;
+    for (int w2 = 0; w2 < warp; ++w2) off += red[w2 * 2 + 1];
+    float pp = off + (incl_sum - bi);              // ||P_i||^2 (exclusive)
     const int t_tok = c * kGT + tid;
     if (t_tok < p.S) {
-        if (p.incl) { dk += g_diag[0]; dv += g_diag[1]; ppk += bk; ppv += bv; }
+        if (p.incl) { d += g_diag; pp += bi; }
         const long long cnt = (p.count_in ? p.count_in[b] : 0ll) + t_tok + (p.incl ? 1 : 0);
-        float cosk = 0.f, cosv = 0.f;
+        float cosv = 0.f;
         if (cnt > 0) {
-            const float s = 1.f / (float)cnt;               // anchor = sum * s
-            cosk = (dk * s) / (fmaxf(sqrtf(g_diag[0]), kNormEps) * fmaxf(sqrtf(fmaxf(ppk, 0.f)) * s, kNormEps));
-            cosv = (dv * s) / (fmaxf(sqrtf(g_diag[1]), kNormEps) * fmaxf(sqrtf(fmaxf(ppv, 0.f)) * s, kNormEps));
+            const float s = 1.f / (float)cnt;      // anchor = sum * s
+            cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pp, 0.f)) * s, kNormEps));
         }
-        const size_t o = ((size_t)b * p.S + t_tok) * p.H + h;
-        p.sim_k[o] = cosk;
-        p.sim_v[o] = cosv;
+        p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = cosv;
     }
 
     tc_fence_before();
@@ -375,7 +355,7 @@ kv_stats_gram_kernel(const GramParams p, const __grid_constant__ CUtensorMap map
         while (clock64() - t0 < 2000000ll) { }
         __syncthreads();
     }
-    if (warp == 1) tmem_dealloc(tmem, kGramTmemCols);
+    if (warp == 1) tmem_dealloc(tmem, kT1TmemCols);
 }
 
 }  // namespace
@@ -391,11 +371,13 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     const int n_chunks = (s.seq + kGT - 1) / kGT;
     const size_t tiles = (size_t)n_chains * (size_t)n_chunks;
     if (tiles == 0) return cudaSuccess;
-    if (tiles > 0x7fffffffu) return cudaErrorInvalidValue;
+    if (2 * tiles > 0x7fffffffu) return cudaErrorInvalidValue;
+    // scratch: per tensor, one 1 KiB record (128 packets of 8 bytes) per tile and one per 8th chunk of a chain
     const size_t anchors = (size_t)n_chains * (size_t)((n_chunks + kGramAnchorEvery - 1) / kGramAnchorEvery);
-    const size_t agg_offset = 256, prefix_offset = agg_offset + tiles * kHeadDim * sizeof(uint4);
-    // (a tag distinguishes this kernel's record layout from the plain kernel's, which may share the scratch)
-    const size_t bytes = ((prefix_offset + anchors * kHeadDim * sizeof(uint4) + 255) / 256 * 256) | 1;
+    const size_t rec = kHeadDim * sizeof(uint2);
+    const size_t agg_offset = 256, prefix_offset = agg_offset + 2 * tiles * rec;
+    // (the low bit distinguishes this kernel's record layout from the plain kernel's, which may share the scratch)
+    const size_t bytes = ((prefix_offset + 2 * anchors * rec + 255) / 256 * 256) | 1;
     if (ws->needs_clear || ws->bytes != bytes || ws->epoch == 0xffffffffu) {
         cudaError_t e = cudaMemsetAsync(ws->ptr, 0, bytes & ~(size_t)1, st);
         if (e != cudaSuccess) return e;
@@ -414,29 +396,28 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
         return cudaErrorNotSupported;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kv_stats_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGramSmem);
+        cudaError_t e = cudaFuncSetAttribute(kv_stats_gram1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kT1Smem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    GramParams gp{};
+    Gram1Params gp{};
     gp.S = s.seq; gp.H = s.n_kv_heads; gp.n_chains = n_chains; gp.n_chunks = n_chunks;
     gp.incl = (p.anchor_mode == TF_ANCHOR_INCL_MEAN);
     if (carry) {
-        gp.sum_k_in = carry->sum_k_in; gp.sum_v_in = carry->sum_v_in;
+        gp.sum_in[0] = carry->sum_k_in; gp.sum_in[1] = carry->sum_v_in;
         gp.count_in = reinterpret_cast<const long long*>(carry->count_in);
-        gp.sum_k_out = carry->sum_k_out; gp.sum_v_out = carry->sum_v_out;
+        gp.sum_out[0] = carry->sum_k_out; gp.sum_out[1] = carry->sum_v_out;
     }
-    gp.sim_k = sim_k; gp.sim_v = sim_v;
+    gp.sim[0] = sim_k; gp.sim[1] = sim_v;
     char* base = static_cast<char*>(ws->ptr);
-    gp.ticket = reinterpret_cast<unsigned int*>(base);
-    gp.ticket_base = ws->ticket_base;
     gp.epoch = ws->epoch;
-    gp.agg_rec = reinterpret_cast<uint4*>(base + agg_offset);
-    gp.prefix_rec = reinterpret_cast<uint4*>(base + prefix_offset);
+    for (int x = 0; x < 2; ++x) {
+        gp.agg_rec[x] = reinterpret_cast<uint2*>(base + agg_offset + x * tiles * rec);
+        gp.prefix_rec[x] = reinterpret_cast<uint2*>(base + prefix_offset + x * anchors * rec);
+    }
     gp.status = ctx->dev_status;
     gp.max_polls = 1 << 20;
-    ws->ticket_base += (unsigned int)tiles;
-    kv_stats_gram_kernel<<<(unsigned)tiles, 128, kGramSmem, st>>>(gp, mk, mv);
+    kv_stats_gram1_kernel<<<(unsigned)(2 * tiles), 128, kT1Smem, st>>>(gp, mk, mv);
     ctx->launches += 1;
     return cudaGetLastError();
 }
