@@ -6,7 +6,10 @@
 // whose key equals it are then taken from the highest index down.  THRESHOLD mode prunes the
 // eligible tokens whose score is strictly above threshold[b] (Alg. 1, "skip if s_KV > tau").
 // The retained positions are compacted in ascending order with warp ballots and a block-wide
-// prefix sum.  Scores are re-read from global memory on each pass (they stay in L1/L2).
+// prefix sum.  For sequences of up to 16384 tokens every thread keeps its scores in registers
+// (token i*1024 + tid in slot i), so the passes run out of registers and shared memory; longer
+// sequences re-read the scores from global memory on each pass.  (Producing the scores inside this
+// kernel as well was measured: one CTA per sequence reads the per-head similarities far too slowly.)
 #include <math_constants.h>
 
 #include "tf_common.cuh"
@@ -55,6 +58,8 @@ __device__ __forceinline__ int block_rank(bool flag, int* s_warp, int& total) {
     return before + __popc(bal & ((1u << lane) - 1u));
 }
 
+// KPT = scores per thread held in registers (0: read them from global memory each time)
+template <int KPT>
 __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectParams p) {
     __shared__ int hist[256];
     __shared__ int s_warp[kSelWarps];
@@ -65,6 +70,22 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     const int b = blockIdx.x, tid = threadIdx.x, S = p.S;
     const float* sc = p.score + (size_t)b * S;
     const uint8_t* el = p.eligible ? p.eligible + (size_t)b * S : nullptr;
+    constexpr int NR = KPT > 0 ? KPT : 1;
+    float sreg[NR];
+    if (KPT > 0) {
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int t = i * kSelThreads + tid;
+            float s = 0.f;
+            if (t < S) {
+                s = sc[t];
+            }
+            sreg[i] = s;
+        }
+    }
+    // score of token t = i*1024 + tid (i is a compile-time index wherever KPT > 0)
+    auto score_at = [&](int i, int t) -> float { return KPT > 0 ? sreg[KPT > 0 ? i : 0] : sc[t]; };
+    constexpr int kChunks = KPT;   // register form: exactly KPT chunks of 1024 tokens
     auto candidate = [&](int t, float s) -> bool {
         return t >= p.warmup && (el == nullptr || el[t] != 0) && s == s;   // NaN never pruned
     };
@@ -80,7 +101,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     } else {
         // E = number of candidates
         int e_local = 0;
-        for (int t = tid; t < S; t += kSelThreads) e_local += candidate(t, sc[t]) ? 1 : 0;
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < NR; ++i) { const int t = i * kSelThreads + tid; e_local += (t < S && candidate(t, score_at(i, t))) ? 1 : 0; }
+        } else {
+            for (int t = tid; t < S; t += kSelThreads) e_local += candidate(t, sc[t]) ? 1 : 0;
+        }
         if (tid == 0) s_count = 0;
         __syncthreads();
         e_local = __reduce_add_sync(0xffffffffu, e_local);
@@ -98,11 +124,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
             for (int shift = 24; shift >= 0; shift -= 8) {
                 for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
                 __syncthreads();
-                for (int t0 = 0; t0 < S; t0 += kSelThreads) {
+#pragma unroll
+                for (int i = 0; i < (KPT > 0 ? kChunks : 1 << 30); ++i) {
+                    const int t0 = i * kSelThreads;
+                    if (KPT == 0 && t0 >= S) break;
                     const int t = t0 + tid;
                     int bin = 256;   // sentinel: this lane adds nothing
                     if (t < S) {
-                        const float s = sc[t];
+                        const float s = score_at(i, t);
                         if (candidate(t, s)) {
                             const unsigned int k = score_key(s);
                             if ((k & mask) == prefix) bin = (int)((k >> shift) & 255u);
@@ -152,10 +181,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     // ---- sweep in index order: decide, count equals, compact ---------------------------------------
     int kept_base = 0, eq_base = 0;
     float th_min = CUDART_INF_F;
-    for (int t0 = 0; t0 < S; t0 += kSelThreads) {
+#pragma unroll
+    for (int i = 0; i < (KPT > 0 ? kChunks : 1 << 30); ++i) {
+        const int t0 = i * kSelThreads;
+        if (t0 >= S) break;
         const int t = t0 + tid;
         const bool in = t < S;
-        const float s = in ? sc[t] : 0.f;
+        const float s = in ? score_at(i, t) : 0.f;
         const bool cand = in && candidate(t, s);
         bool prune = false;
         if (p.mode == TF_SELECT_THRESHOLD) {
@@ -194,6 +226,18 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     }
 }
 
+namespace {
+cudaError_t launch_select_form(const SelectParams& sp, int batch, cudaStream_t st) {
+    const dim3 grid(batch), block(kSelThreads);
+    const int S = sp.S;
+    if (S <= 2 * kSelThreads) return launch_dependent(select_kernel<2>, grid, block, 0, st, sp);
+    if (S <= 4 * kSelThreads) return launch_dependent(select_kernel<4>, grid, block, 0, st, sp);
+    if (S <= 8 * kSelThreads) return launch_dependent(select_kernel<8>, grid, block, 0, st, sp);
+    if (S <= 16 * kSelThreads) return launch_dependent(select_kernel<16>, grid, block, 0, st, sp);
+    return launch_dependent(select_kernel<0>, grid, block, 0, st, sp);
+}
+}  // namespace
+
 cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                           const float* score, uint8_t* keep_mask, int32_t* kept_idx,
                           int32_t* n_kept, float* theta, cudaStream_t st) {
@@ -203,7 +247,7 @@ cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params
     sp.S = s.seq; sp.warmup = p.warmup_tokens; sp.mode = p.select_mode;
     sp.p_target = (long long)floor(p.prune_ratio * (double)s.seq);
     sp.keep_mask = keep_mask; sp.kept_idx = kept_idx; sp.n_kept = n_kept; sp.theta = theta;
-    cudaError_t e = launch_dependent(select_kernel, dim3(s.batch), dim3(kSelThreads), 0, st, sp);
+    cudaError_t e = launch_select_form(sp, s.batch, st);
     ctx->launches += 1;
     return e;
 }
