@@ -719,7 +719,7 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     const double ctas_shared = (double)s.batch * s.n_q_heads * ceil(s.seq * kept_frac / (kQTiles * kTileM));
     int sms = 148;
     { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
-    const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 0.75 * sms);
+    const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 1.0 * sms);
     const int rows_per_cta = split ? kTileM : kQTiles * kTileM;
     tp.n_row_blocks = (s.seq + rows_per_cta - 1) / rows_per_cta;
     const double kv_bytes = 2.0 * s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
