@@ -91,14 +91,19 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def attention_flops(kept_idx: np.ndarray, n_kept: np.ndarray, Hq: int, d: int, window: int) -> float:
-    """4*d*Hq * sum over retained tokens of the number of visible keys (the work actually needed)."""
+def attention_flops(kept_idx: np.ndarray, n_kept: np.ndarray, Hq: int, d: int, window: int, retained_only: bool = False) -> float:
+    """4*d*Hq * sum over retained tokens of the number of visible keys (the work actually needed).
+    retained_only: a retained query sees retained tokens only (TF_KV_RETAINED)."""
     tot = 0.0
     for b in range(kept_idx.shape[0]):
         t = kept_idx[b, : n_kept[b]].astype(np.int64)
-        vis = t + 1
-        if window > 0:
-            vis = np.minimum(vis, window)
+        if retained_only:
+            first = np.searchsorted(t, t - window + 1) if window > 0 else np.zeros_like(t)
+            vis = np.arange(t.size) - first + 1
+        else:
+            vis = t + 1
+            if window > 0:
+                vis = np.minimum(vis, window)
         tot += float(vis.sum())
     return 4.0 * d * Hq * tot
 
@@ -185,10 +190,50 @@ def run_reference(args, wl):
     print(json.dumps(out))
 
 
+def run_decode(args, wl, tfb, dev, local):
+    """Online decode step (Algorithm 1 per token + threshold feedback + single-query attention): B sequences,
+    a cache of seq tokens of the workload's layer-0 K/V, the new token at the last position.  Not the headline
+    metric; one JSON line of its own."""
+    _, q, k, v = next(wl.layer_qkv([0], dev))
+    B, S, Hq, d = q.shape
+    Hkv = k.shape[2]
+    ctx = tfb.Context(local)
+    params = tfb.default_params(prune_ratio=args.prune, warmup_tokens=4)
+    st = tfb.DecodeState(B, Hkv, dev, tau0=10.0)      # a threshold no score reaches: every step pays the attention
+    shape = tfb.make_shape(None, k, v, window=wl.window, n_q_heads=Hq)
+    O = torch.empty(B, Hq, d, dtype=q.dtype, device=dev)
+    shape.q_stride[:] = [q.stride(0), 0, q.stride(2)]
+    shape.o_stride[:] = [O.stride(0), 0, O.stride(1)]
+    pos = torch.full((B,), S - 1, dtype=torch.int32, device=dev)
+    score = torch.empty(B, device=dev); skip = torch.empty(B, dtype=torch.uint8, device=dev)
+    for _ in range(max(3, args.warmup)):
+        ctx.tf_decode_step(shape, params, 0.0, q[:, S - 1], k, v, pos, st, O, score, skip)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ctx.tf_decode_step(shape, params, 0.0, q[:, S - 1], k, v, pos, st, O, score, skip)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    pk, pk_kind = peaks()
+    vis = min(S, wl.window) if wl.window > 0 else S
+    cache_bytes = 2.0 * B * Hkv * vis * d * q.element_size()          # K and V rows one query group reads once
+    print(json.dumps({"metric": "online decode steps/s per layer (no skip, cache = seq tokens)", "value": B / (ms * 1e-3),
+                      "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "bf16" if q.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+                      "config": workload_config(wl, args), "gpu_launches": 2 * args.steps,
+                      "roofline": {"kernel": "decode_attention", "bound": "hbm", "achieved": cache_bytes / (ms * 1e-3) / 1e9,
+                                   "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": cache_bytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                                   "traffic": None, "peak_kind": pk_kind, "algorithmic_per_launch": cache_bytes}}))
+    ctx.close()
+
+
 def workload_config(wl, args):
     return {"workload": f"{wl.name}: {wl.stack.name if wl.stack else 'llama2-7b head shape'} one layer, batch {wl.batch}, "
                         f"seq {wl.seq}, {wl.n_q_heads} q heads / {wl.n_kv_heads} kv heads, head_dim 128, "
-                        f"{'bf16' if wl.dtype == torch.bfloat16 else 'fp32'}, window {wl.window}, prune {args.prune}",
+                        f"{'bf16' if wl.dtype == torch.bfloat16 else 'fp32'}, window {wl.window}, prune {args.prune}"
+                        + (", retained keys only" if getattr(args, "kv_visibility", "all") == "retained" else ""),
             "global_batch": wl.batch * args.gpus, "seq_len": wl.seq, "prune_ratio": args.prune,
             "parallelism": f"replicas x{args.gpus} (independent sequences, no collective)",
             "l2": "inputs rotate over distinct layers whose total size exceeds the 126 MB L2"}
@@ -203,6 +248,10 @@ def main():
     ap.add_argument("--prune", type=float, default=0.5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv-visibility", default="all", choices=["all", "retained"],
+                    help="retained: kept queries attend kept keys only (a different, smaller computation)")
+    ap.add_argument("--decode", action="store_true",
+                    help="measure the online decode step (one new token per sequence against a cache of seq tokens) instead")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -225,6 +274,9 @@ def main():
     wl.seed += 7919 * rank
 
     tfb.lib()   # fails loudly if the CUDA library is not built
+    if args.decode:
+        run_decode(args, wl, tfb, dev, local)
+        return
     ring = make_ring(wl, dev, min_bytes=300 << 20)
     B, S, Hq, d = ring[0][0].shape
     Hkv = ring[0][1].shape[2]
@@ -232,7 +284,8 @@ def main():
     ctx = tfb.Context(local)
     O = torch.empty_like(ring[0][0])
     shape = tfb.make_shape(ring[0][0], ring[0][1], ring[0][2], O, window=wl.window)
-    params = tfb.default_params(prune_ratio=args.prune, warmup_tokens=4)
+    params = tfb.default_params(prune_ratio=args.prune, warmup_tokens=4,
+                                kv_visibility=tfb.TF_KV_RETAINED if args.kv_visibility == "retained" else tfb.TF_KV_ALL)
     ctx.ensure_workspace(shape, params)
     sim_k = torch.empty(B, S, Hkv, device=dev); sim_v = torch.empty_like(sim_k)
     score = torch.empty(B, S, device=dev)
@@ -285,7 +338,8 @@ def main():
         ctx.tf_score_fuse(shape, params, sk, sv, sc)
         ctx.tf_select(shape, params, sc, keep, ix, n_)
         torch.cuda.synchronize()
-        flops += attention_flops(ix.cpu().numpy(), n_.cpu().numpy(), Hq, d, wl.window) / len(ring)
+        flops += attention_flops(ix.cpu().numpy(), n_.cpu().numpy(), Hq, d, wl.window,
+                                 args.kv_visibility == "retained") / len(ring)
         state.append((sk, sv, sc, ix, n_))
 
     def stage(name, i):
@@ -368,7 +422,7 @@ def main():
                "vs_baseline": None, "dtype": "bf16" if wl.dtype == torch.bfloat16 else "f32", "data": "synthetic",
                "config": workload_config(wl, args), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                "roofline": roof, "kernels": kern}
-        if not args.no_cpu_baseline and world == 1:
+        if not args.no_cpu_baseline and world == 1 and args.kv_visibility == "all":   # the baseline arm times the default reading
             q, k, v = ring[0]
             out["cpu_baseline"] = oracle_sample(wl, (q.float().cpu().numpy(), k.float().cpu().numpy(),
                                                      v.float().cpu().numpy()), args.prune)
