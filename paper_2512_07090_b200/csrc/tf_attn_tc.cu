@@ -699,6 +699,14 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
             e = cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Cfg<true>::kSmemBytes);
         if (e != cudaSuccess) return e;
+        // The kernel moves registers from its third warpgroup to the softmax warpgroups (setmaxnreg: 168 -> 72
+        // releases 128 x 96, 168 -> 216 takes 256 x 48).  An inc only receives what a dec of the same CTA
+        // released and waits for it without limit, so the trade must balance: refuse to launch a build that
+        // does not start at 168 registers per thread.
+        cudaFuncAttributes fa{};
+        if (cudaFuncGetAttributes(&fa, attention_tc_kernel<false>) != cudaSuccess || fa.numRegs != 168 ||
+            cudaFuncGetAttributes(&fa, attention_tc_kernel<true>) != cudaSuccess || fa.numRegs != 168)
+            return cudaErrorNotSupported;
         attr_set = true;
     }
     TcParams tp{};
