@@ -229,6 +229,20 @@ def run_decode(args, wl, tfb, dev, local):
     ctx.close()
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Every rank of an N-GPU run works on its own replica of the workload (sequences are independent)."""
+    return seed + 7919 * rank
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """A multi-rank run is as slow as its slowest rank."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def workload_config(wl, args):
     return {"workload": f"{wl.name}: {wl.stack.name if wl.stack else 'llama2-7b head shape'} one layer, batch {wl.batch}, "
                         f"seq {wl.seq}, {wl.n_q_heads} q heads / {wl.n_kv_heads} kv heads, head_dim 128, "
@@ -271,7 +285,7 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
-    wl.seed += 7919 * rank
+    wl.seed = rank_seed(wl.seed, rank)
 
     tfb.lib()   # fails loudly if the CUDA library is not built
     if args.decode:
@@ -363,10 +377,7 @@ def main():
         per[n] = s0.elapsed_time(s1) / args.steps
     clocks = sampler.stop()
 
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     tokens_per_step = B * S * world
     value = tokens_per_step * args.steps / (ms * 1e-3)
 
@@ -387,10 +398,7 @@ def main():
     f1.record()
     sync_all()
     e2e_ms = f0.elapsed_time(f1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     e2e = {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": int((qh.numel() + kh.numel() + vh.numel()) * es),
            "d2h_bytes_per_step": int(oh.numel() * es + nh.numel() * 4), "steps": e2e_steps}
