@@ -11,6 +11,8 @@
 //   over cache positions <= pos (optionally windowed) unless the token is skipped, in which case
 //   its output row is zero (Section 3.2).  The 8 warps take interleaved blocks of 32 keys, each
 //   with its own online softmax; the partial results are merged through shared memory.
+#include <algorithm>
+
 #include "tf_common.cuh"
 
 namespace tf {
@@ -207,6 +209,191 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_attention_kernel(const 
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// bf16 decode attention for grouped heads: one CTA per (split of the visible keys, KV head, sequence)
+// serves all G query heads of the group, so K and V rows are read once per group.  16 lanes share a
+// key row (16-byte loads, two adjacent rows per warp instruction); the 16 half-warps of the CTA take
+// keys 16 apart, four at a time, each with its own online softmax; half-warps are merged through
+// shuffles and shared memory.  With more than one split the CTA leaves (max, sum, unnormalised
+// output) per head in scratch and decode_combine_kernel merges the splits.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kDecBatch = 4;          // keys a half-warp scores before it updates its running maximum
+constexpr int kPartialFloats = kHeadDim + 2;
+
+struct DecGqaParams {
+    const __nv_bfloat16* Q; const __nv_bfloat16* K; const __nv_bfloat16* V; __nv_bfloat16* O;
+    long long q_b, q_h, o_b, o_h;
+    Strides3 ks, vs;
+    const int32_t* pos; const uint8_t* skip;
+    int Hq, Hkv, window, n_splits;
+    float scale_log2;
+    float* partial;                   // [B][Hq][n_splits][130] when n_splits > 1
+};
+
+__device__ __forceinline__ void unpack8(const uint4& r, float* f) {
+    f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+    f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+    f[4] = __uint_as_float(r.z << 16); f[5] = __uint_as_float(r.z & 0xffff0000u);
+    f[6] = __uint_as_float(r.w << 16); f[7] = __uint_as_float(r.w & 0xffff0000u);
+}
+
+template <int G>
+__global__ void __launch_bounds__(256) decode_attention_gqa_kernel(const DecGqaParams p) {
+    __shared__ float part_s[8][G][kPartialFloats];
+    grid_dependency_wait();
+    const int split = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
+    if (p.skip[b]) {
+        if (split == 0 && p.n_splits == 1)
+            for (int i = threadIdx.x; i < G * kHeadDim; i += 256)
+                p.O[(long long)b * p.o_b + (long long)(kh * G + i / kHeadDim) * p.o_h + (i % kHeadDim)] = __float2bfloat16_rn(0.f);
+        return;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+    const int t = p.pos[b];
+    const int j_lo = (p.window > 0) ? max(0, t - p.window + 1) : 0;
+    const int n_vis = t - j_lo + 1;
+    const int per = ((n_vis + p.n_splits - 1) / p.n_splits + 15) / 16 * 16;     // keys per split, a multiple of 16
+    const int k_lo = j_lo + split * per, k_hi = min(t + 1, k_lo + per);           // [k_lo, k_hi)
+
+    float q[G][8];
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        float f[8];
+        unpack8(ldg16(p.Q + (long long)b * p.q_b + (long long)(kh * G + h) * p.q_h + l16 * 8), f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) q[h][e] = f[e] * p.scale_log2;
+    }
+    const __nv_bfloat16* Kb = p.K + (long long)b * p.ks.b + (long long)kh * p.ks.h + l16 * 8;
+    const __nv_bfloat16* Vb = p.V + (long long)b * p.vs.b + (long long)kh * p.vs.h + l16 * 8;
+
+    float m[G], l[G], acc[G][8];
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        m[h] = -1e30f; l[h] = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[h][e] = 0.f;
+    }
+    // half-warp hw = 2 warp + half takes keys k_lo + hw + 16 i.  The loop bound is the warp's (its lower half-warp's):
+    // both halves must make the same number of trips because the shuffles below name all 32 lanes; a key index
+    // past the end is handled by the (j < k_hi) predicates.
+    for (int kb = k_lo + warp * 2; kb < k_hi; kb += 16 * kDecBatch) {
+        const int k0 = kb + half;
+        uint4 kr[kDecBatch], vr[kDecBatch];
+#pragma unroll
+        for (int u = 0; u < kDecBatch; ++u) {
+            const int j = k0 + 16 * u;
+            kr[u] = (j < k_hi) ? ldg16(Kb + (long long)j * p.ks.t) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < kDecBatch; ++u) {
+            const int j = k0 + 16 * u;
+            vr[u] = (j < k_hi) ? ldg16(Vb + (long long)j * p.vs.t) : make_uint4(0, 0, 0, 0);
+        }
+        float s[G][kDecBatch];
+#pragma unroll
+        for (int u = 0; u < kDecBatch; ++u) {
+            float kf[8];
+            unpack8(kr[u], kf);
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; e += 2) { d0 = fmaf(q[h][e], kf[e], d0); d1 = fmaf(q[h][e + 1], kf[e + 1], d1); }
+                float d = d0 + d1;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);   // stays inside the half-warp
+                s[h][u] = (k0 + 16 * u < k_hi) ? d : -1e30f;
+            }
+        }
+        float corr[G], pw[G][kDecBatch];
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            float mx = m[h];
+#pragma unroll
+            for (int u = 0; u < kDecBatch; ++u) mx = fmaxf(mx, s[h][u]);
+            corr[h] = exp2f(m[h] - mx);
+            float ps = 0.f;
+#pragma unroll
+            for (int u = 0; u < kDecBatch; ++u) {
+                pw[h][u] = (k0 + 16 * u < k_hi) ? exp2f(s[h][u] - mx) : 0.f;
+                ps += pw[h][u];
+            }
+            l[h] = fmaf(l[h], corr[h], ps);
+            m[h] = mx;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[h][e] *= corr[h];
+        }
+#pragma unroll
+        for (int u = 0; u < kDecBatch; ++u) {
+            float vf[8];
+            unpack8(vr[u], vf);
+#pragma unroll
+            for (int h = 0; h < G; ++h)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[h][e] = fmaf(pw[h][u], vf[e], acc[h][e]);
+        }
+    }
+    // ---- merge: the two half-warps of a warp by shuffle, the 8 warps through shared memory ---------------
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        const float mo = __shfl_xor_sync(0xffffffffu, m[h], 16), lo = __shfl_xor_sync(0xffffffffu, l[h], 16);
+        const float mm = fmaxf(m[h], mo);
+        const float c_me = exp2f(m[h] - mm), c_ot = exp2f(mo - mm);
+        l[h] = l[h] * c_me + lo * c_ot;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float ao = __shfl_xor_sync(0xffffffffu, acc[h][e], 16);
+            acc[h][e] = acc[h][e] * c_me + ao * c_ot;
+        }
+        m[h] = mm;
+        if (half == 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) part_s[warp][h][l16 * 8 + e] = acc[h][e];
+            if (l16 == 0) { part_s[warp][h][kHeadDim] = m[h]; part_s[warp][h][kHeadDim + 1] = l[h]; }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < G * kHeadDim; i += 256) {
+        const int h = i / kHeadDim, d = i % kHeadDim;
+        float M = -1e30f;
+#pragma unroll
+        for (int w2 = 0; w2 < 8; ++w2) M = fmaxf(M, part_s[w2][h][kHeadDim]);
+        float L = 0.f, o = 0.f;
+#pragma unroll
+        for (int w2 = 0; w2 < 8; ++w2) {
+            const float c = exp2f(part_s[w2][h][kHeadDim] - M);
+            L = fmaf(part_s[w2][h][kHeadDim + 1], c, L);
+            o = fmaf(part_s[w2][h][d], c, o);
+        }
+        const int qh = kh * G + h;
+        if (p.n_splits == 1) {
+            p.O[(long long)b * p.o_b + (long long)qh * p.o_h + d] = __float2bfloat16_rn(o / L);
+        } else {
+            float* dst = p.partial + (((size_t)b * p.Hq + qh) * p.n_splits + split) * kPartialFloats;
+            dst[d] = o;
+            if (d == 0) { dst[kHeadDim] = M; dst[kHeadDim + 1] = L; }
+        }
+    }
+}
+
+// merges the splits of one (query head, sequence); a skipped token gets its zero row here
+__global__ void __launch_bounds__(kHeadDim) decode_combine_kernel(const DecGqaParams p) {
+    grid_dependency_wait();
+    const int qh = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
+    __nv_bfloat16* out = p.O + (long long)b * p.o_b + (long long)qh * p.o_h + d;
+    if (p.skip[b]) { *out = __float2bfloat16_rn(0.f); return; }
+    const float* src = p.partial + ((size_t)b * p.Hq + qh) * p.n_splits * kPartialFloats;
+    float M = -1e30f;
+    for (int s2 = 0; s2 < p.n_splits; ++s2) M = fmaxf(M, src[s2 * kPartialFloats + kHeadDim]);
+    float L = 0.f, o = 0.f;
+    for (int s2 = 0; s2 < p.n_splits; ++s2) {
+        const float c = exp2f(src[s2 * kPartialFloats + kHeadDim] - M);
+        L = fmaf(src[s2 * kPartialFloats + kHeadDim + 1], c, L);
+        o = fmaf(src[s2 * kPartialFloats + d], c, o);
+    }
+    *out = __float2bfloat16_rn(o / L);
+}
+
 cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const tf_decode_args& a,
                                cudaStream_t st) {
     if (s.batch == 0) return cudaSuccess;
@@ -235,6 +422,40 @@ cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_p
     ap.Hq = s.n_q_heads; ap.Hkv = s.n_kv_heads; ap.window = s.window;
     const float scale = s.softmax_scale != 0.f ? s.softmax_scale : 1.f / sqrtf((float)s.head_dim);
     ap.scale_log2 = scale * 1.4426950408889634f;
+    // bf16 with 1, 2, 4 or 8 query heads per KV head: the grouped kernel (K / V read once per group), split
+    // over the visible keys when that is needed to fill the GPU and the bound workspace can hold the partials
+    const int G = s.n_q_heads / s.n_kv_heads;
+    if (s.dtype == TF_BF16 && (G == 1 || G == 2 || G == 4 || G == 8) && (s.q_stride[2] % 8 == 0) && (s.q_stride[0] % 8 == 0) &&
+        (reinterpret_cast<uintptr_t>(a.q_new) & 15u) == 0) {
+        DecGqaParams gp{};
+        gp.Q = static_cast<const __nv_bfloat16*>(a.q_new); gp.K = static_cast<const __nv_bfloat16*>(a.K_cache);
+        gp.V = static_cast<const __nv_bfloat16*>(a.V_cache); gp.O = static_cast<__nv_bfloat16*>(a.O_new);
+        gp.q_b = ap.q_b; gp.q_h = ap.q_h; gp.o_b = ap.o_b; gp.o_h = ap.o_h;
+        gp.ks = ap.ks; gp.vs = ap.vs; gp.pos = a.pos; gp.skip = a.skip_out;
+        gp.Hq = s.n_q_heads; gp.Hkv = s.n_kv_heads; gp.window = s.window; gp.scale_log2 = ap.scale_log2;
+        int sms = 148;
+        { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+        const int max_keys = s.window > 0 ? (s.window < s.seq ? s.window : s.seq) : s.seq;   // pos is device data: size for the worst case
+        int n_splits = (2 * sms + s.batch * s.n_kv_heads - 1) / (s.batch * s.n_kv_heads);
+        n_splits = std::max(1, std::min(n_splits, max_keys / 512));                             // at least 512 keys per split
+        const size_t need = (size_t)s.batch * s.n_q_heads * n_splits * kPartialFloats * sizeof(float);
+        if (n_splits > 1 && (!ctx->workspace || ctx->workspace_bytes < need)) n_splits = 1;
+        gp.n_splits = n_splits;
+        gp.partial = n_splits > 1 ? static_cast<float*>(ctx->workspace) : nullptr;
+        const dim3 grid((unsigned)n_splits, (unsigned)s.n_kv_heads, (unsigned)s.batch);
+        switch (G) {
+            case 1: e = launch_dependent(decode_attention_gqa_kernel<1>, grid, dim3(256), 0, st, gp); break;
+            case 2: e = launch_dependent(decode_attention_gqa_kernel<2>, grid, dim3(256), 0, st, gp); break;
+            case 4: e = launch_dependent(decode_attention_gqa_kernel<4>, grid, dim3(256), 0, st, gp); break;
+            default: e = launch_dependent(decode_attention_gqa_kernel<8>, grid, dim3(256), 0, st, gp); break;
+        }
+        ctx->launches += 1;
+        if (e == cudaSuccess && n_splits > 1) {
+            e = launch_dependent(decode_combine_kernel, dim3((unsigned)s.n_q_heads, (unsigned)s.batch), dim3(kHeadDim), 0, st, gp);
+            ctx->launches += 1;
+        }
+        return e;
+    }
     const dim3 grid((unsigned)s.n_q_heads, (unsigned)s.batch);
     if (s.dtype == TF_BF16) e = launch_dependent(decode_attention_kernel<__nv_bfloat16>, grid, dim3(kDecWarps * 32), 0, st, ap);
     else                    e = launch_dependent(decode_attention_kernel<float>, grid, dim3(kDecWarps * 32), 0, st, ap);

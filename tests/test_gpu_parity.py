@@ -312,14 +312,18 @@ def test_device_rejects_bad_arguments_without_launching():
 
 
 # ------------------------------------------------------------------------------- online decode step
-@pytest.mark.parametrize("dtype,mode,window", [(torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0), (torch.float32, tfb.TF_ANCHOR_PAST_MEAN, 40),
-                                               (torch.bfloat16, tfb.TF_ANCHOR_EMA, 0), (torch.bfloat16, tfb.TF_ANCHOR_INCL_MEAN, 0)])
-def test_decode_steps_match_oracle(dtype, mode, window):
+@pytest.mark.parametrize("dtype,mode,window,S0,T,Hq,Hkv",
+                         [(torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0, 70, 90, 8, 2), (torch.float32, tfb.TF_ANCHOR_PAST_MEAN, 40, 70, 90, 8, 2),
+                          (torch.bfloat16, tfb.TF_ANCHOR_EMA, 0, 70, 90, 8, 2), (torch.bfloat16, tfb.TF_ANCHOR_INCL_MEAN, 0, 70, 90, 8, 2),
+                          # long caches: the grouped kernel splits the keys over several CTAs and merges the partial results
+                          (torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0, 2900, 24, 8, 1), (torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 1500, 2100, 24, 4, 4),
+                          (torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0, 1100, 24, 6, 3)])
+def test_decode_steps_match_oracle(dtype, mode, window, S0, T, Hq, Hkv):
     """A prefill of 70 tokens seeds the anchors through tf_kv_stats' carry; then 90 decode steps run in
     lockstep with the oracle: scores within 1e-5, thresholds within 1e-6, skip decisions equal unless the
     score is within 1e-5 of the threshold (then the oracle's state is forced on so the runs stay comparable),
     outputs within the attention tolerance; skipped rows are zero."""
-    B, S0, T, Hq, Hkv = 2, 70, 90, 8, 2
+    B = 2
     S = S0 + T
     q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=123, dup=0.4)
     qn, kn, vn = oracle_inputs(q, k, v)
@@ -367,6 +371,6 @@ def test_decode_steps_match_oracle(dtype, mode, window):
     code, det = ctx.tf_get_status()
     assert code == tfb.TF_OK, det
     assert np.array_equal(st.count.cpu().numpy(), ost["count"]) and np.array_equal(st.steps.cpu().numpy(), ost["steps"])
-    assert 0 < n_skips < B * T            # the case exercises both branches
+    assert 0 < n_skips < B * T            # the case exercises both branches (skip and attend)
     assert near <= 2
     ctx.close()
