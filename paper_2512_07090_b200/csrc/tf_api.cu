@@ -394,7 +394,7 @@ tf_status tf_set_attention_path(tf_ctx* ctx, int use_tensor_cores) {
 }
 
 tf_status tf_set_scan_path(tf_ctx* ctx, int path) {
-    if (!ctx || path < 0 || path > 2) return TF_ERR_INVALID_ARG;
+    if (!ctx || path < 0 || path > 3) return TF_ERR_INVALID_ARG;
     ctx->scan_path = path;
     return TF_OK;
 }

@@ -304,7 +304,7 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
                             const tf_carry* carry, ScanScratch* ws, cudaStream_t st) {
     if (ctx->scan_path != 1 && kv_stats_gram_usable(s, p))
         return launch_kv_stats_gram(ctx, s, p, K, V, sim_k, sim_v, carry, ws, st);
-    if (ctx->scan_path == 2) return cudaErrorNotSupported;
+    if (ctx->scan_path >= 2) return cudaErrorNotSupported;
     const ScanPlan pl = scan_plan(s);
     const size_t tiles = (size_t)pl.n_chains * (size_t)pl.n_chunks;
     if (tiles == 0) return cudaSuccess;

@@ -18,6 +18,8 @@
 // share an SM, so that the loads of some overlap the arithmetic of others.  Carries travel through tagged
 // records with the same fixed-association look-back as the plain kernel (see tf_scan.cu); a record is 128
 // 8-byte packets {value, tag}.  All waits are bounded.
+#include <algorithm>
+
 #include "tf_ptx.cuh"
 
 namespace tf {
@@ -358,6 +360,287 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     if (warp == 1) tmem_dealloc(tmem, kT1TmemCols);
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Persistent form: one CTA per SM with six workers of 128 threads; every worker takes tiles from an atomic
+// ticket (chunk index slowest, so the records a tile waits for belong to tickets drawn before its own) and
+// runs the sequence above on its own 36 KiB of shared memory and its own 80 TMEM columns.  What it changes:
+//  * barriers, the small operand and TMEM are set up once per SM instead of once per tile;
+//  * the tensor pipe takes ~53 cycles for any M=128 product of up to 80 columns, and with six tiles in flight
+//    that pipe, not HBM, is what the one-tile kernel saturates.  Here the small operand lies directly behind
+//    each 64-dim block of the tile, so that rows 64..143 of the block are "rows 64-127 of X, then c1 c2 c3":
+//    the second half of G and X C are ONE product of 80 columns (24 products per tile instead of 32);
+//  * X^T 1 and the first half of G are issued together, the look-back loads go out under them, and the next
+//    tile's TMA load starts as soon as the last product has read the current one, under the scan and cosine.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kPWorkers = 6;
+constexpr int kPThreads = kPWorkers * 128;
+constexpr int kPBlock = kHalf + 16 * 128;                            // [128 tile rows + 16 small-operand rows][128 B]
+constexpr int kPWorkerBytes = 2 * kPBlock;                           // 36 KiB: dims 0-63, dims 64-127
+constexpr int kPOffMisc = kPWorkers * kPWorkerBytes;
+constexpr int kPMiscPerWorker = 96;                                  // 3 mbarriers, next ticket, scan scratch
+constexpr int kPSmem = kPOffMisc + kPWorkers * kPMiscPerWorker + 64;
+constexpr uint32_t kPTmemCols = 512;                                 // worker w: columns 80 w .. 80 w + 79
+constexpr uint32_t kPNoTile = 0xffffffffu;
+constexpr uint32_t kIdescG80 = idesc(80, false);
+constexpr int kPLookBack = kGramAnchorEvery - 1;                     // aggregates between a prefix record and a tile
+
+struct GramPParams {
+    Gram1Params g;
+    unsigned int* ticket; unsigned int ticket_base, n_tiles;        // n_tiles counts (tile, tensor) pairs
+};
+
+__device__ __forceinline__ void worker_sync(int w) { asm volatile("bar.sync %0, 128;" :: "r"(w + 1) : "memory"); }
+// byte offset, from the worker's base, of element (row n, index k) of the small operand
+__device__ __forceinline__ uint32_t pbt_off(int n, int k) {
+    return (uint32_t)((k >> 6) * kPBlock + kHalf + n * 128 + ((((k & 63) >> 3) ^ (n & 7)) << 4) + (k & 7) * 2);
+}
+__device__ __forceinline__ uint64_t pdesc_mnmajor(uint32_t addr) {   // next 64 MN elements one block later
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(kPBlock >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
+__global__ void __launch_bounds__(kPThreads, 1)
+kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CUtensorMap mapK,
+                                const __grid_constant__ CUtensorMap mapV) {
+    extern __shared__ uint8_t smem[];
+    const Gram1Params& p = pp.g;
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {
+        if (threadIdx.x == 0) report_error(p.status, TF_ERR_TIMEOUT, 299);
+        return;
+    }
+    const int tid = threadIdx.x & 127, w = threadIdx.x >> 7, warp = tid >> 5, lane = tid & 31;
+    uint8_t* misc = smem + kPOffMisc + w * kPMiscPerWorker;
+    const uint32_t bar_tma = smem_u32(misc), bar_small = bar_tma + 8, bar_g = bar_tma + 16;
+    volatile unsigned int* s_next = reinterpret_cast<volatile unsigned int*>(misc + 24);
+    float* red = reinterpret_cast<float*>(misc + 32);                 // [4 warps][2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPOffMisc + kPWorkers * kPMiscPerWorker);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint8_t* my = smem + w * kPWorkerBytes;
+    const uint32_t xa = sbase + w * kPWorkerBytes;
+
+    if (tid == 0) {
+        mbar_init(bar_tma, 1);
+        mbar_init(bar_small, 1);
+        mbar_init(bar_g, 1);
+        if (w == 0) *abort_flag = 0;
+        mbar_fence_init();
+    }
+    // small operand (16 rows behind each 64-dim block): rows 0-2 take the carry, row 6 is all ones, the rest 0
+    {
+        uint8_t* dst = my + (tid >> 6) * kPBlock + kHalf + (tid & 63) * 32;
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(dst + 16) = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    *reinterpret_cast<unsigned short*>(my + pbt_off(6, tid)) = 0x3f80;
+    if (threadIdx.x < 32) tmem_alloc(smem_u32(tmem_slot), kPTmemCols);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tm_g = tmem + 80u * w, tm_s = tm_g + 64u;                       // G half / small product
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+
+    auto issue_load = [&](unsigned int t) {                                         // worker thread 0 only
+        const unsigned int tile = t >> 1;
+        const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
+        const CUtensorMap* map = (t & 1) ? &mapV : &mapK;
+        mbar_expect_tx(bar_tma, kXBytes);
+        tma_load_4d(xa, map, bar_tma, 0, chain % p.H, c * kGT, chain / p.H);
+        tma_load_4d(xa + kPBlock, map, bar_tma, 64, chain % p.H, c * kGT, chain / p.H);
+    };
+    auto draw = [&]() -> unsigned int {
+        const unsigned int t = atomicAdd(pp.ticket, 1u) - pp.ticket_base;
+        return t < pp.n_tiles ? t : kPNoTile;
+    };
+
+    if (tid == 0) {
+        const unsigned int t0 = draw();
+        *s_next = t0;
+        if (t0 != kPNoTile) issue_load(t0);
+    }
+    worker_sync(w);
+    unsigned int t = *s_next;
+    uint32_t tile_phase = 0;          // bar_tma and bar_small complete once per tile, bar_g twice
+
+    while (t != kPNoTile) {
+        const int x = (int)(t & 1u);
+        const unsigned int tile = t >> 1;
+        const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
+        const int b = chain / p.H, h = chain % p.H;
+        uint2* agg_rec = p.agg_rec[x];
+        uint2* prefix_rec = p.prefix_rec[x];
+        unsigned int t_next = kPNoTile;
+        if (tid == 0) t_next = draw();                       // the answer is needed only when this tile's products are done
+
+        wait_bar(bar_tma, tile_phase, abort_flag, p.status, 200);
+
+        // ---- X^T 1 (columns 64-79) and columns 0-63 of G, issued together ------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)                   // 16 tokens per step
+                mma_ss(tm_s, pdesc_mnmajor(xa + kk * 16 * 128), desc_kmajor(xa + (kk >> 2) * kPBlock + kHalf + (kk & 3) * 32),
+                       kIdescAgg, kk > 0);
+            mma_commit(bar_small);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {                 // 16 dims per step
+                const uint32_t off = (kk >> 2) * kPBlock + (kk & 3) * 32;
+                mma_ss(tm_g, desc_kmajor(xa + off), desc_kmajor(xa + off), kIdescG64, kk > 0);
+            }
+            mma_commit(bar_g);
+        }
+        // ---- look-back requests go out under the products (thread = dim) -------------------------------------------
+        const int a0 = c > 0 ? ((c - 1) / kGramAnchorEvery) * kGramAnchorEvery : 0;
+        const uint2* prec = prefix_rec + ((size_t)(a0 / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid;
+        const uint2* arec = agg_rec + ((size_t)a0 * p.n_chains + chain) * kHeadDim + tid;    // chunk a0 + u: u n_chains records on
+        const size_t astride = (size_t)p.n_chains * kHeadDim;
+        uint2 pfirst = make_uint2(0, 0), afirst[kPLookBack + 1];
+        if (c > 0) {
+            pfirst = ld_packet2(prec);
+#pragma unroll
+            for (int u = 0; u <= kPLookBack; ++u)
+                if (a0 + u < c) afirst[u] = ld_packet2(arec + u * astride);
+        }
+
+        wait_bar(bar_small, tile_phase, abort_flag, p.status, 201);
+        tile_phase ^= 1;
+        tc_fence_after();
+        float agg;
+        {
+            uint32_t r0[8];
+            tmem_ld8(tm_s + lane_off, r0);
+            tmem_wait_ld();
+            agg = __uint_as_float(r0[6]);
+        }
+        if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, p.epoch);
+
+        // ---- carry: prefix record of chunk a0 + aggregates of chunks a0 .. c-1, in ascending order ---------------------
+        float carry = 0.f;
+        if (c == 0) {
+            if (p.sum_in[x]) carry = p.sum_in[x][(size_t)chain * kHeadDim + tid];
+        } else {
+            float A = 0.f;
+#pragma unroll
+            for (int u = 0; u <= kPLookBack; ++u)
+                if (a0 + u < c) A += wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile);
+            carry = wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile) + A;
+        }
+        if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
+            st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, p.epoch);
+        if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = carry + agg;
+        {   // the carry as c1 + c2 + c3 (bf16 each) into rows 0-2 of the small operand
+            float cr = carry;
+#pragma unroll
+            for (int n = 0; n < 3; ++n) {
+                const unsigned short hb = bf16_bits(cr);
+                *reinterpret_cast<unsigned short*>(my + pbt_off(n, tid)) = hb;
+                cr -= __uint_as_float((uint32_t)hb << 16);
+            }
+        }
+        float c2 = warp_sum(carry * carry);            // ||C||^2 (worker-wide sum over dims)
+        if (lane == 0) red[warp * 2] = c2;
+
+        // thread i adds row i of a 64-column half of G left of the diagonal
+        float r_sum = 0.f, g_diag = 0.f;
+        auto add_half = [&](int hh) {
+#pragma unroll
+            for (int lc = 0; lc < 2; ++lc) {
+                const int cb = 2 * hh + lc;               // 32-column block of G (warp-uniform comparisons)
+                if (cb > warp) continue;
+                uint32_t g[32];
+                tmem_ld32(tm_g + lane_off + lc * 32, g);
+                tmem_wait_ld();
+                if (cb < warp) {
+                    float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) s4[e & 3] += __uint_as_float(g[e]);
+                    r_sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const float v = __uint_as_float(g[e]);
+                        r_sum += (e < lane) ? v : 0.f;
+                        g_diag = (e == lane) ? v : g_diag;
+                    }
+                }
+            }
+        };
+        wait_bar(bar_g, 0, abort_flag, p.status, 202);
+        tc_fence_after();
+        add_half(0);
+        fence_proxy_async();
+        tc_fence_before();
+        worker_sync(w);
+        c2 = (red[0] + red[2]) + (red[4] + red[6]);
+        // ---- columns 64-127 of G and u = X [c1 c2 c3 ..]^T as one product of 80 columns ------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t off = (kk >> 2) * kPBlock + (kk & 3) * 32;
+                mma_ss(tm_g, desc_kmajor(xa + off), desc_kmajor(xa + 64 * 128 + off), kIdescG80, kk > 0);
+            }
+            mma_commit(bar_g);
+        }
+        wait_bar(bar_g, 1, abort_flag, p.status, 203);
+        tc_fence_after();
+        // every product that reads this tile has completed: the next one may land on it
+        if (tid == 0) {
+            if (*abort_flag) t_next = kPNoTile;
+            *s_next = t_next;
+            if (t_next != kPNoTile) issue_load(t_next);
+        }
+        add_half(1);
+        float d;
+        {
+            uint32_t r0[8];
+            tmem_ld8(tm_s + lane_off, r0);
+            tmem_wait_ld();
+            d = (__uint_as_float(r0[0]) + __uint_as_float(r0[1])) + __uint_as_float(r0[2]) + r_sum;   // <x_i, P_i>
+        }
+
+        // ---- ||P_i||^2 by a worker-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosine -------------
+        const float bi = fmaf(2.f, d, g_diag);
+        float incl_sum = bi;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float n = __shfl_up_sync(0xffffffffu, incl_sum, o);
+            if (lane >= o) incl_sum += n;
+        }
+        if (lane == 31) red[warp * 2 + 1] = incl_sum;
+        tc_fence_before();
+        worker_sync(w);
+        float off = c2;
+        for (int w2 = 0; w2 < warp; ++w2) off += red[w2 * 2 + 1];
+        float pn = off + (incl_sum - bi);              // ||P_i||^2 (exclusive)
+        const int t_tok = c * kGT + tid;
+        if (t_tok < p.S) {
+            if (p.incl) { d += g_diag; pn += bi; }
+            const long long cnt = (p.count_in ? p.count_in[b] : 0ll) + t_tok + (p.incl ? 1 : 0);
+            float cosv = 0.f;
+            if (cnt > 0) {
+                const float s = 1.f / (float)cnt;
+                cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pn, 0.f)) * s, kNormEps));
+            }
+            p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = cosv;
+        }
+        t = *s_next;      // rewritten, like red[], only after the next tile's first worker barrier
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) { }
+        __syncthreads();
+    }
+    if (threadIdx.x < 32) tmem_dealloc(tmem, kPTmemCols);
+}
+
 }  // namespace
 
 bool kv_stats_gram_usable(const tf_shape& s, const tf_filter_params& p) {
@@ -417,6 +700,27 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     }
     gp.status = ctx->dev_status;
     gp.max_polls = 1 << 20;
+    if (ctx->scan_path == 3) {
+        static bool attr_set_p = false;
+        if (!attr_set_p) {
+            cudaError_t e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
+            if (e != cudaSuccess) return e;
+            attr_set_p = true;
+        }
+        int sms = 148;
+        { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+        const unsigned int n_work = (unsigned int)(2 * tiles);
+        const unsigned int grid = std::min<unsigned int>((unsigned int)sms, (n_work + kPWorkers - 1) / kPWorkers);
+        GramPParams pp{};
+        pp.g = gp;
+        pp.ticket = reinterpret_cast<unsigned int*>(base);
+        pp.ticket_base = ws->ticket_base;
+        pp.n_tiles = n_work;
+        ws->ticket_base += n_work + grid * kPWorkers;      // every worker draws once past the end
+        kv_stats_gram_persistent_kernel<<<grid, kPThreads, kPSmem, st>>>(pp, mk, mv);
+        ctx->launches += 1;
+        return cudaGetLastError();
+    }
     kv_stats_gram1_kernel<<<(unsigned)(2 * tiles), 128, kT1Smem, st>>>(gp, mk, mv);
     ctx->launches += 1;
     return cudaGetLastError();
