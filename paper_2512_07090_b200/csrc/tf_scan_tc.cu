@@ -390,6 +390,28 @@ struct GramPParams {
     unsigned int* ticket; unsigned int ticket_base, n_tiles;        // n_tiles counts (tile, tensor) pairs
 };
 
+// mbarrier wait for the persistent kernel: the hardware may park the thread for up to the hinted time per try, and
+// the clock and the abort flag are looked at once per 32 tries, so a waiting warp costs few issue slots
+__device__ __forceinline__ bool wait_bar_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevStatus* status,
+                                                unsigned long long where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            uint32_t ok;
+            asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
+                         : "=r"(ok) : "r"(bar), "r"(parity), "r"(100000u) : "memory");
+            if (ok) return true;
+        }
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kGramWaitCycles) {
+            *abort_flag = 1;
+            report_error(status, TF_ERR_TIMEOUT, where);
+            return false;
+        }
+    }
+}
 __device__ __forceinline__ void worker_sync(int w) { asm volatile("bar.sync %0, 128;" :: "r"(w + 1) : "memory"); }
 // byte offset, from the worker's base, of element (row n, index k) of the small operand
 __device__ __forceinline__ uint32_t pbt_off(int n, int k) {
@@ -413,8 +435,8 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
     const int tid = threadIdx.x & 127, w = threadIdx.x >> 7, warp = tid >> 5, lane = tid & 31;
     uint8_t* misc = smem + kPOffMisc + w * kPMiscPerWorker;
     const uint32_t bar_tma = smem_u32(misc), bar_small = bar_tma + 8, bar_g = bar_tma + 16;
-    volatile unsigned int* s_next = reinterpret_cast<volatile unsigned int*>(misc + 24);
-    float* red = reinterpret_cast<float*>(misc + 32);                 // [4 warps][2]
+    volatile unsigned int* s_next = reinterpret_cast<volatile unsigned int*>(misc + 32);   // next tile: {chunk, chain, sequence, head | tensor << 30}
+    float* red = reinterpret_cast<float*>(misc + 48);                 // [4 warps][2]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPOffMisc + kPWorkers * kPMiscPerWorker);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     uint8_t* my = smem + w * kPWorkerBytes;
@@ -444,39 +466,42 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
     const uint32_t tm_g = tmem + 80u * w, tm_s = tm_g + 64u;                       // G half / small product
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
 
-    auto issue_load = [&](unsigned int t) {                                         // worker thread 0 only
+    // worker thread 0 only: decodes ticket t for everyone (the divisions are done once, off the critical path),
+    // leaves the result in shared memory and starts the tile's load
+    auto announce_and_load = [&](unsigned int t) {
+        if (t == kPNoTile) {
+            s_next[0] = kPNoTile;
+            return;
+        }
         const unsigned int tile = t >> 1;
-        const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
+        const unsigned int c = tile / (unsigned)p.n_chains, chain = tile - c * (unsigned)p.n_chains;
+        const unsigned int b = chain / (unsigned)p.H, h = chain - b * (unsigned)p.H;
+        s_next[0] = c; s_next[1] = chain; s_next[2] = b; s_next[3] = h | ((t & 1u) << 30);
         const CUtensorMap* map = (t & 1) ? &mapV : &mapK;
         mbar_expect_tx(bar_tma, kXBytes);
-        tma_load_4d(xa, map, bar_tma, 0, chain % p.H, c * kGT, chain / p.H);
-        tma_load_4d(xa + kPBlock, map, bar_tma, 64, chain % p.H, c * kGT, chain / p.H);
+        tma_load_4d(xa, map, bar_tma, 0, (int)h, (int)c * kGT, (int)b);
+        tma_load_4d(xa + kPBlock, map, bar_tma, 64, (int)h, (int)c * kGT, (int)b);
     };
     auto draw = [&]() -> unsigned int {
         const unsigned int t = atomicAdd(pp.ticket, 1u) - pp.ticket_base;
         return t < pp.n_tiles ? t : kPNoTile;
     };
 
-    if (tid == 0) {
-        const unsigned int t0 = draw();
-        *s_next = t0;
-        if (t0 != kPNoTile) issue_load(t0);
-    }
+    if (tid == 0) announce_and_load(draw());
     worker_sync(w);
-    unsigned int t = *s_next;
+    uint4 cur = make_uint4(s_next[0], s_next[1], s_next[2], s_next[3]);
     uint32_t tile_phase = 0;          // bar_tma and bar_small complete once per tile, bar_g twice
 
-    while (t != kPNoTile) {
-        const int x = (int)(t & 1u);
-        const unsigned int tile = t >> 1;
-        const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
-        const int b = chain / p.H, h = chain % p.H;
+    while (cur.x != kPNoTile) {
+        const int c = (int)cur.x, chain = (int)cur.y, b = (int)cur.z, h = (int)(cur.w & 0x3fffffffu), x = (int)(cur.w >> 30);
+        const unsigned int tile = (unsigned)c * (unsigned)p.n_chains + (unsigned)chain;
         uint2* agg_rec = p.agg_rec[x];
         uint2* prefix_rec = p.prefix_rec[x];
         unsigned int t_next = kPNoTile;
         if (tid == 0) t_next = draw();                       // the answer is needed only when this tile's products are done
+        const long long cnt0 = p.count_in ? p.count_in[b] : 0ll;
 
-        wait_bar(bar_tma, tile_phase, abort_flag, p.status, 200);
+        wait_bar_parked(bar_tma, tile_phase, abort_flag, p.status, 200);
 
         // ---- X^T 1 (columns 64-79) and columns 0-63 of G, issued together ------------------------------------
         if (tid == 0) {
@@ -506,7 +531,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
                 if (a0 + u < c) afirst[u] = ld_packet2(arec + u * astride);
         }
 
-        wait_bar(bar_small, tile_phase, abort_flag, p.status, 201);
+        wait_bar_parked(bar_small, tile_phase, abort_flag, p.status, 201);
         tile_phase ^= 1;
         tc_fence_after();
         float agg;
@@ -569,7 +594,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
                 }
             }
         };
-        wait_bar(bar_g, 0, abort_flag, p.status, 202);
+        wait_bar_parked(bar_g, 0, abort_flag, p.status, 202);
         tc_fence_after();
         add_half(0);
         fence_proxy_async();
@@ -586,14 +611,10 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             }
             mma_commit(bar_g);
         }
-        wait_bar(bar_g, 1, abort_flag, p.status, 203);
+        wait_bar_parked(bar_g, 1, abort_flag, p.status, 203);
         tc_fence_after();
         // every product that reads this tile has completed: the next one may land on it
-        if (tid == 0) {
-            if (*abort_flag) t_next = kPNoTile;
-            *s_next = t_next;
-            if (t_next != kPNoTile) issue_load(t_next);
-        }
+        if (tid == 0) announce_and_load(*abort_flag ? kPNoTile : t_next);
         add_half(1);
         float d;
         {
@@ -620,15 +641,21 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         const int t_tok = c * kGT + tid;
         if (t_tok < p.S) {
             if (p.incl) { d += g_diag; pn += bi; }
-            const long long cnt = (p.count_in ? p.count_in[b] : 0ll) + t_tok + (p.incl ? 1 : 0);
+            const long long cnt = cnt0 + t_tok + (p.incl ? 1 : 0);
             float cosv = 0.f;
             if (cnt > 0) {
-                const float s = 1.f / (float)cnt;
-                cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pn, 0.f)) * s, kNormEps));
+                // anchor = sum / cnt; the 1 / cnt cancels unless a norm falls under its clamp
+                const float fc = (float)cnt, lim = kNormEps * kNormEps;
+                if (g_diag > lim && pn > lim * fc * fc) {
+                    cosv = d * rsqrtf(g_diag) * rsqrtf(pn);
+                } else {
+                    const float s = 1.f / fc;
+                    cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pn, 0.f)) * s, kNormEps));
+                }
             }
             p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = cosv;
         }
-        t = *s_next;      // rewritten, like red[], only after the next tile's first worker barrier
+        cur = make_uint4(s_next[0], s_next[1], s_next[2], s_next[3]);   // rewritten, like red[], only after the next tile's first worker barrier
     }
 
     tc_fence_before();
