@@ -19,6 +19,7 @@
 // records with the same fixed-association look-back as the plain kernel (see tf_scan.cu); a record is 128
 // 8-byte packets {value, tag}.  All waits are bounded.
 #include <algorithm>
+#include <utility>
 
 #include "tf_ptx.cuh"
 
@@ -390,6 +391,25 @@ struct GramPParams {
     unsigned int* ticket; unsigned int ticket_base, n_tiles;        // n_tiles counts (tile, tensor) pairs
 };
 
+// Eight products of one accumulation chain.  The operand descriptors differ only in the 14-bit address field of
+// their low word, so the issuing thread adds compile-time offsets (units of 16 bytes) to two precomputed low
+// words instead of rebuilding 64-bit descriptors per product: issue is on the critical path of every tile.
+template <uint32_t A_OFF, uint32_t B_OFF, bool ACC>
+__device__ __forceinline__ void mma_step(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t id) {
+    asm volatile("{\n.reg .pred p;\n.reg .b32 ta, tb;\n.reg .b64 da, db;\n"
+                 "setp.ne.b32 p, %6, 0;\n"
+                 "add.u32 ta, %1, %7;\nadd.u32 tb, %3, %8;\n"
+                 "mov.b64 da, {ta, %2};\nmov.b64 db, {tb, %4};\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
+                 :: "r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(id), "n"(ACC ? 1 : 0), "n"(A_OFF), "n"(B_OFF)
+                 : "memory");
+}
+__host__ __device__ constexpr uint32_t kmaj_step(int kk, int block_bytes) { return (uint32_t)(((kk >> 2) * block_bytes + (kk & 3) * 32) >> 4); }
+template <int BLOCK, bool A_MN, int... KK>
+__device__ __forceinline__ void mma_burst(std::integer_sequence<int, KK...>, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi,
+                                          uint32_t b_lo, uint32_t b_hi, uint32_t id) {
+    (mma_step<(A_MN ? (uint32_t)(KK * 16 * 128 >> 4) : kmaj_step(KK, BLOCK)), kmaj_step(KK, BLOCK), (KK > 0)>(d_tmem, a_lo, a_hi, b_lo, b_hi, id), ...);
+}
 // mbarrier wait for the persistent kernel: the hardware may park the thread for up to the hinted time per try, and
 // the clock and the abort flag are looked at once per 32 tries, so a waiting warp costs few issue slots
 __device__ __forceinline__ bool wait_bar_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevStatus* status,
@@ -465,6 +485,12 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
     const uint32_t tmem = *tmem_slot;
     const uint32_t tm_g = tmem + 80u * w, tm_s = tm_g + 64u;                       // G half / small product
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    // operand descriptor words (see desc_kmajor / pdesc_mnmajor): address field of this worker's tile, the two
+    // leading-dimension fields, and the high word (8-row groups 1024 B apart, version 1, 128-byte swizzle)
+    const uint32_t x_lo = (xa & 0x3ffffu) >> 4;
+    constexpr uint32_t dlo_k = 1u << 16, dlo_mn = (uint32_t)(kPBlock >> 4) << 16;
+    constexpr uint32_t dhi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+    constexpr std::make_integer_sequence<int, 8> k8{};
 
     // worker thread 0 only: decodes ticket t for everyone (the divisions are done once, off the critical path),
     // leaves the result in shared memory and starts the tile's load
@@ -506,16 +532,9 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         // ---- X^T 1 (columns 64-79) and columns 0-63 of G, issued together ------------------------------------
         if (tid == 0) {
             tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)                   // 16 tokens per step
-                mma_ss(tm_s, pdesc_mnmajor(xa + kk * 16 * 128), desc_kmajor(xa + (kk >> 2) * kPBlock + kHalf + (kk & 3) * 32),
-                       kIdescAgg, kk > 0);
+            mma_burst<kPBlock, true>(k8, tm_s, x_lo | dlo_mn, dhi, x_lo + (kHalf >> 4) | dlo_k, dhi, kIdescAgg);   // 16 tokens per step
             mma_commit(bar_small);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {                 // 16 dims per step
-                const uint32_t off = (kk >> 2) * kPBlock + (kk & 3) * 32;
-                mma_ss(tm_g, desc_kmajor(xa + off), desc_kmajor(xa + off), kIdescG64, kk > 0);
-            }
+            mma_burst<kPBlock, false>(k8, tm_g, x_lo | dlo_k, dhi, x_lo | dlo_k, dhi, kIdescG64);               // 16 dims per step
             mma_commit(bar_g);
         }
         // ---- look-back requests go out under the products (thread = dim) -------------------------------------------
@@ -604,11 +623,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         // ---- columns 64-127 of G and u = X [c1 c2 c3 ..]^T as one product of 80 columns ------------------------------------
         if (tid == 0) {
             tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t off = (kk >> 2) * kPBlock + (kk & 3) * 32;
-                mma_ss(tm_g, desc_kmajor(xa + off), desc_kmajor(xa + 64 * 128 + off), kIdescG80, kk > 0);
-            }
+            mma_burst<kPBlock, false>(k8, tm_g, x_lo | dlo_k, dhi, x_lo + (64 * 128 >> 4) | dlo_k, dhi, kIdescG80);
             mma_commit(bar_g);
         }
         wait_bar_parked(bar_g, 1, abort_flag, p.status, 203);
