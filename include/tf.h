@@ -238,9 +238,11 @@ tf_status tf_clear_status(tf_ctx *ctx);
  * tile per CTA with its K/V tiles split between the CTA's two softmax groups.  For A/B checks. */
 tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
 
-/* Which kernel tf_kv_stats uses: 0 = choose (default), 1 = the plain CUDA-core kernel (any dtype and
- * anchor mode), 2 = the kernel that forms 128-token Gram matrices on the tensor cores (bf16,
- * running-sum anchors; other calls then fail with TF_ERR_CUDA).  For A/B checks. */
+/* Which kernel tf_kv_stats uses: 0 = choose (default: by dtype, anchor mode and problem size), 1 = the
+ * plain CUDA-core kernel (any dtype and anchor mode), 2 = the kernel that forms 128-token Gram matrices
+ * on the tensor cores, one tile per CTA, 3 = the same arithmetic as a persistent kernel (one CTA per SM,
+ * six tiles in flight).  2 and 3 take bf16 with running-sum anchors; other calls then fail with
+ * TF_ERR_CUDA.  For A/B checks. */
 tf_status tf_set_scan_path(tf_ctx *ctx, int path);
 
 const char *tf_status_string(tf_status s);

@@ -239,7 +239,7 @@ class Context:
         _check(lib().tf_set_attention_path(self._h, C.c_int(int(path))), "tf_set_attention_path")
 
     def tf_set_scan_path(self, path: int):
-        """0: choose; 1: plain CUDA-core similarity scan; 2: Gram-matrix scan on the tensor cores (bf16 sums)."""
+        """0: choose; 1: plain CUDA-core similarity scan; 2: Gram-matrix scan on the tensor cores (bf16 sums), one tile per CTA; 3: the same, persistent."""
         _check(lib().tf_set_scan_path(self._h, C.c_int(int(path))), "tf_set_scan_path")
 
     @property

@@ -121,7 +121,7 @@ struct tf_ctx {
     tf::ScanScratch scan_user;     // scan bookkeeping of the caller's workspace
     tf::ScanScratch scan_owned;    // ... and of owned_ws
     int use_tensor_cores;          // bf16 attention path
-    int scan_path;                 // tf_kv_stats: 0 = choose, 1 = plain CUDA-core kernel, 2 = Gram-matrix kernel (bf16 sums)
+    int scan_path;                 // tf_kv_stats: 0 = choose, 1 = plain CUDA-core kernel, 2 / 3 = Gram-matrix kernel, one tile per CTA / persistent
     int attention_form;            // tensor-core kernel: 0 = choose by grid size, 1 = shared K/V tiles, 2 = split K/V tiles
     long long launches;            // kernels launched through this context
     // tf_layer_filter_host staging (owned, grown on demand)

@@ -30,7 +30,7 @@ constexpr int kGT = 128;                       // tokens per tile
 constexpr int kHalf = 128 * 128;               // one [128 rows][128 B] swizzled block
 constexpr int kXBytes = 2 * kHalf;             // one tensor's tile
 constexpr int kBtBytes = 2 * 16 * 128;         // small B operand: [16 rows][128 elements], two 64-element blocks
-constexpr int kGramAnchorEvery = 8;
+constexpr int kGramAnchorEvery = 4;             // a prefix record every 4th chunk: at most 4 aggregates + 1 prefix per look-back
 constexpr int kGramPollBatch = 4;
 constexpr long long kGramWaitCycles = 1000000000ll;
 
@@ -742,15 +742,18 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     }
     gp.status = ctx->dev_status;
     gp.max_polls = 1 << 20;
-    if (ctx->scan_path == 3) {
+    int sms = 148;
+    { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+    // the persistent form pays its set-up once per SM and wins once every worker sees several tiles (measured
+    // cross-over between 2.3 and 11.5 tiles per worker); below that the one-tile-per-CTA form starts sooner
+    const bool persistent = ctx->scan_path == 3 || (ctx->scan_path == 0 && 2 * tiles >= (size_t)4 * sms * kPWorkers);
+    if (persistent) {
         static bool attr_set_p = false;
         if (!attr_set_p) {
             cudaError_t e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
             if (e != cudaSuccess) return e;
             attr_set_p = true;
         }
-        int sms = 148;
-        { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
         const unsigned int n_work = (unsigned int)(2 * tiles);
         const unsigned int grid = std::min<unsigned int>((unsigned int)sms, (n_work + kPWorkers - 1) / kPWorkers);
         GramPParams pp{};
