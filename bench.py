@@ -421,9 +421,14 @@ def main():
             kern["pruned_attention"].update(bound="alu", achieved=ach, unit="TFLOP/s", peak=148 * 128 * 2 * 1.965e-3,
                                             frac=ach / (148 * 128 * 2 * 1.965e-3))
         dom = max(names, key=lambda n: per[n])
+        # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the ncu
+        # captures summarised under profiles/ (50 % pruning, all keys visible); None where none was taken.
+        ncu_traffic = {("c2", "pruned_attention"): 42046208 + 91136, ("c3", "pruned_attention"): 420643840 + 154753536,
+                       ("c3", "kv_stats"): 337320704 + 17053696, ("c2", "kv_stats"): 33894144}
+        traffic = ncu_traffic.get((wl.name, dom)) if (args.prune == 0.5 and args.kv_visibility == "all") else None
         roof = {"kernel": dom, "bound": kern[dom].get("bound", "latency"), "achieved": kern[dom].get("achieved"),
                 "peak": kern[dom].get("peak"), "unit": kern[dom].get("unit"), "frac": kern[dom].get("frac"),
-                "traffic": None, "peak_kind": f"{pk_kind} ({'sustained' if long_run else 'burst'} bf16)" if dom == "pruned_attention" else pk_kind,
+                "traffic": traffic, "peak_kind": f"{pk_kind} ({'sustained' if long_run else 'burst'} bf16)" if dom == "pruned_attention" else pk_kind,
                 "algorithmic_per_launch": flops if dom == "pruned_attention" else kv_bytes}
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
