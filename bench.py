@@ -204,12 +204,14 @@ def run_decode(args, wl, tfb, dev, local):
     O = torch.empty(B, Hq, d, dtype=q.dtype, device=dev)
     shape.q_stride[:] = [q.stride(0), 0, q.stride(2)]
     shape.o_stride[:] = [O.stride(0), 0, O.stride(1)]
+    ctx.ensure_workspace(shape, params)               # the decode step keeps its split-key partial results there
     pos = torch.full((B,), S - 1, dtype=torch.int32, device=dev)
     score = torch.empty(B, device=dev); skip = torch.empty(B, dtype=torch.uint8, device=dev)
     for _ in range(max(3, args.warmup)):
         ctx.tf_decode_step(shape, params, 0.0, q[:, S - 1], k, v, pos, st, O, score, skip)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launches
     e0.record()
     for _ in range(args.steps):
         ctx.tf_decode_step(shape, params, 0.0, q[:, S - 1], k, v, pos, st, O, score, skip)
@@ -222,7 +224,7 @@ def run_decode(args, wl, tfb, dev, local):
     print(json.dumps({"metric": "online decode steps/s per layer (no skip, cache = seq tokens)", "value": B / (ms * 1e-3),
                       "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
                       "higher_is_better": True, "dtype": "bf16" if q.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-                      "config": workload_config(wl, args), "gpu_launches": 2 * args.steps,
+                      "config": workload_config(wl, args), "gpu_launches": int(ctx.launches - launches0),
                       "roofline": {"kernel": "decode_attention", "bound": "hbm", "achieved": cache_bytes / (ms * 1e-3) / 1e9,
                                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": cache_bytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
                                    "traffic": None, "peak_kind": pk_kind, "algorithmic_per_launch": cache_bytes}}))

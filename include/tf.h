@@ -210,7 +210,10 @@ typedef struct {
  *          and head strides of q_new [B, n_q_heads, 128], o_stride[0], o_stride[2] those of O_new.
  *   pos:   device int32 [B], 0 <= pos[b] < seq, the cache row that already holds the current token.
  *   score (may be NULL) fp32 [B]; skip u8 [B] (required): 1 = attention skipped, O_new row is zero.
- * Two launches on the stream; the state is advanced in place. */
+ * Two or three launches on the stream; the state is advanced in place.  If a workspace is bound
+ * (tf_set_workspace, any size tf_workspace_bytes returns for a prefill of this shape is enough: the
+ * need is batch * n_q_heads * splits * 520 bytes), bf16 calls split the visible keys over several CTAs
+ * per KV head and keep their partial results there; without one each KV head is one CTA. */
 tf_status tf_decode_step(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
                          float eta, int32_t alg1_sign, const void *q_new, const void *K_cache,
                          const void *V_cache, const int32_t *pos, const tf_decode_state *state,

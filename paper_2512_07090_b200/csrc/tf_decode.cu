@@ -211,13 +211,25 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_attention_kernel(const 
 
 // ---------------------------------------------------------------------------------------------------
 // bf16 decode attention for grouped heads: one CTA per (split of the visible keys, KV head, sequence)
-// serves all G query heads of the group, so K and V rows are read once per group.  16 lanes share a
-// key row (16-byte loads, two adjacent rows per warp instruction); the 16 half-warps of the CTA take
-// keys 16 apart, four at a time, each with its own online softmax; half-warps are merged through
-// shuffles and shared memory.  With more than one split the CTA leaves (max, sum, unnormalised
-// output) per head in scratch and decode_combine_kernel merges the splits.
+// serves all G <= 8 query heads of the group, so K and V rows are read once per group.  The two small
+// products run on warp-level tensor-core instructions (m16n8k16, bf16 in, fp32 out): the path is
+// bandwidth-bound, and the CUDA-core dot products (8 FMAs and 4 shuffles per (head, key)) were what kept
+// it from the bandwidth, so the point is the instruction count, not the flops.  Per warp and block of
+// 16 keys:
+//   S^T[16 keys x 8 heads] = K_blk Q^T     8 products over the 128 dims.  A dot product does not care in
+//                                           which order the dims are visited, so lane (g, t) loads 16-byte
+//                                           pieces t, t+4, t+8, t+12 of its two key rows (g, g+8) and of
+//                                           query head g, and both operands use the same dim order: no
+//                                           shared memory, no shuffles, every load a full 16 bytes;
+//   online softmax on the accumulator layout (lane holds keys g, g+8 for heads 2t, 2t+1: the maximum
+//   over keys is three shuffles); P^T goes back through two 8x8 register transposes (movmatrix);
+//   O^T[128 dims x 8 heads] += V_blk^T P^T  8 products.  Lane (g, t) loads dims 16g..16g+15 of its four
+//                                           key rows (2t, 2t+1, 2t+8, 2t+9); the pairs "same dim, two
+//                                           consecutive keys" the A operand wants are byte permutes.
+// The 8 warps take key blocks 8 apart, each with its own online softmax; they are merged through shared
+// memory.  With more than one split the CTA leaves (max, sum, unnormalised output) per head in scratch
+// and decode_combine_kernel merges the splits.
 // ---------------------------------------------------------------------------------------------------
-constexpr int kDecBatch = 4;          // keys a half-warp scores before it updates its running maximum
 constexpr int kPartialFloats = kHeadDim + 2;
 
 struct DecGqaParams {
@@ -230,15 +242,22 @@ struct DecGqaParams {
     float* partial;                   // [B][Hq][n_splits][130] when n_splits > 1
 };
 
-__device__ __forceinline__ void unpack8(const uint4& r, float* f) {
-    f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
-    f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
-    f[4] = __uint_as_float(r.z << 16); f[5] = __uint_as_float(r.z & 0xffff0000u);
-    f[6] = __uint_as_float(r.w << 16); f[7] = __uint_as_float(r.w & 0xffff0000u);
+__device__ __forceinline__ void mma_bf16_16816(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ uint32_t transpose8x8_b16(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
+}
+__device__ __forceinline__ uint32_t word_of(const uint4& r, int w) { return w == 0 ? r.x : w == 1 ? r.y : w == 2 ? r.z : r.w; }
 
 template <int G>
-__global__ void __launch_bounds__(256) decode_attention_gqa_kernel(const DecGqaParams p) {
+__global__ void __launch_bounds__(256, 2) decode_attention_gqa_kernel(const DecGqaParams p) {
     __shared__ float part_s[8][G][kPartialFloats];
     grid_dependency_wait();
     const int split = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
@@ -248,108 +267,100 @@ __global__ void __launch_bounds__(256) decode_attention_gqa_kernel(const DecGqaP
                 p.O[(long long)b * p.o_b + (long long)(kh * G + i / kHeadDim) * p.o_h + (i % kHeadDim)] = __float2bfloat16_rn(0.f);
         return;
     }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
-    const int t = p.pos[b];
-    const int j_lo = (p.window > 0) ? max(0, t - p.window + 1) : 0;
-    const int n_vis = t - j_lo + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int t_pos = p.pos[b];
+    const int j_lo = (p.window > 0) ? max(0, t_pos - p.window + 1) : 0;
+    const int n_vis = t_pos - j_lo + 1;
     const int per = ((n_vis + p.n_splits - 1) / p.n_splits + 15) / 16 * 16;     // keys per split, a multiple of 16
-    const int k_lo = j_lo + split * per, k_hi = min(t + 1, k_lo + per);           // [k_lo, k_hi)
+    const int k_lo = j_lo + split * per, k_hi = min(t_pos + 1, k_lo + per);       // [k_lo, k_hi)
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
 
-    float q[G][8];
+    // Q^T as the B operand of the 8 score products: head g, pieces t + 4i; product 2i + u takes words 2u, 2u + 1
+    uint32_t qb[8][2];
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-        float f[8];
-        unpack8(ldg16(p.Q + (long long)b * p.q_b + (long long)(kh * G + h) * p.q_h + l16 * 8), f);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) q[h][e] = f[e] * p.scale_log2;
+    for (int i = 0; i < 4; ++i) {
+        const uint4 r = (g < G) ? ldg16(p.Q + (long long)b * p.q_b + (long long)(kh * G + g) * p.q_h + 8 * (t + 4 * i)) : zero4;
+        qb[2 * i][0] = r.x; qb[2 * i][1] = r.y; qb[2 * i + 1][0] = r.z; qb[2 * i + 1][1] = r.w;
     }
-    const __nv_bfloat16* Kb = p.K + (long long)b * p.ks.b + (long long)kh * p.ks.h + l16 * 8;
-    const __nv_bfloat16* Vb = p.V + (long long)b * p.vs.b + (long long)kh * p.vs.h + l16 * 8;
+    const __nv_bfloat16* Kb = p.K + (long long)b * p.ks.b + (long long)kh * p.ks.h;
+    const __nv_bfloat16* Vb = p.V + (long long)b * p.vs.b + (long long)kh * p.vs.h + 16 * g;
 
-    float m[G], l[G], acc[G][8];
+    // this lane's part of the state: heads 2t and 2t + 1 (m is the same in all lanes of equal t; l is the lane's share)
+    float m[2] = {-1e30f, -1e30f}, l[2] = {0.f, 0.f};
+    float o[8][4];                                   // O^T: product mt, rows (dims) 16g + mt and 16g + 8 + mt, columns (heads) 2t, 2t + 1
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-        m[h] = -1e30f; l[h] = 0.f;
+    for (int mt = 0; mt < 8; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
+
+    for (int kb = k_lo + 16 * warp; kb < k_hi; kb += 16 * 8) {       // warp-uniform bounds: the shuffles below name all lanes
+        uint4 kr[2][4], vr[4][2];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[h][e] = 0.f;
-    }
-    // half-warp hw = 2 warp + half takes keys k_lo + hw + 16 i.  The loop bound is the warp's (its lower half-warp's):
-    // both halves must make the same number of trips because the shuffles below name all 32 lanes; a key index
-    // past the end is handled by the (j < k_hi) predicates.
-    for (int kb = k_lo + warp * 2; kb < k_hi; kb += 16 * kDecBatch) {
-        const int k0 = kb + half;
-        uint4 kr[kDecBatch], vr[kDecBatch];
+        for (int h = 0; h < 2; ++h) {
+            const int j = kb + g + 8 * h;
 #pragma unroll
-        for (int u = 0; u < kDecBatch; ++u) {
-            const int j = k0 + 16 * u;
-            kr[u] = (j < k_hi) ? ldg16(Kb + (long long)j * p.ks.t) : make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < 4; ++i) kr[h][i] = (j < k_hi) ? ldg16(Kb + (long long)j * p.ks.t + 8 * (t + 4 * i)) : zero4;
         }
 #pragma unroll
-        for (int u = 0; u < kDecBatch; ++u) {
-            const int j = k0 + 16 * u;
-            vr[u] = (j < k_hi) ? ldg16(Vb + (long long)j * p.vs.t) : make_uint4(0, 0, 0, 0);
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const int j = kb + 2 * t + (q4 & 1) + 8 * (q4 >> 1);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) vr[q4][i] = (j < k_hi) ? ldg16(Vb + (long long)j * p.vs.t + 8 * i) : zero4;
         }
-        float s[G][kDecBatch];
+        // ---- scores: rows = keys g, g + 8; columns = heads 2t, 2t + 1 -----------------------------------------
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int u = 0; u < kDecBatch; ++u) {
-            float kf[8];
-            unpack8(kr[u], kf);
-#pragma unroll
-            for (int h = 0; h < G; ++h) {
-                float d0 = 0.f, d1 = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; e += 2) { d0 = fmaf(q[h][e], kf[e], d0); d1 = fmaf(q[h][e + 1], kf[e + 1], d1); }
-                float d = d0 + d1;
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);   // stays inside the half-warp
-                s[h][u] = (k0 + 16 * u < k_hi) ? d : -1e30f;
-            }
+        for (int i = 0; i < 4; ++i) {
+            mma_bf16_16816(s, kr[0][i].x, kr[1][i].x, kr[0][i].y, kr[1][i].y, qb[2 * i][0], qb[2 * i][1]);
+            mma_bf16_16816(s, kr[0][i].z, kr[1][i].z, kr[0][i].w, kr[1][i].w, qb[2 * i + 1][0], qb[2 * i + 1][1]);
         }
-        float corr[G], pw[G][kDecBatch];
+        const bool v0 = kb + g < k_hi, v1 = kb + g + 8 < k_hi;
+        s[0] = v0 ? s[0] * p.scale_log2 : -1e30f; s[1] = v0 ? s[1] * p.scale_log2 : -1e30f;
+        s[2] = v1 ? s[2] * p.scale_log2 : -1e30f; s[3] = v1 ? s[3] * p.scale_log2 : -1e30f;
+        float corr[2], pr[4];
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-            float mx = m[h];
-#pragma unroll
-            for (int u = 0; u < kDecBatch; ++u) mx = fmaxf(mx, s[h][u]);
-            corr[h] = exp2f(m[h] - mx);
-            float ps = 0.f;
-#pragma unroll
-            for (int u = 0; u < kDecBatch; ++u) {
-                pw[h][u] = (k0 + 16 * u < k_hi) ? exp2f(s[h][u] - mx) : 0.f;
-                ps += pw[h][u];
-            }
-            l[h] = fmaf(l[h], corr[h], ps);
-            m[h] = mx;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[h][e] *= corr[h];
+        for (int c = 0; c < 2; ++c) {
+            float mx = fmaxf(s[c], s[c + 2]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float mn = fmaxf(m[c], mx);
+            corr[c] = exp2f(m[c] - mn);
+            m[c] = mn;
+            pr[c] = v0 ? exp2f(s[c] - mn) : 0.f;
+            pr[c + 2] = v1 ? exp2f(s[c + 2] - mn) : 0.f;
+            l[c] = fmaf(l[c], corr[c], pr[c] + pr[c + 2]);
         }
+        // P^T (keys x heads) -> the B operand wants head g with keys 2t, 2t+1 / 2t+8, 2t+9: two 8x8 transposes
+        const uint32_t pb0 = transpose8x8_b16(pack_bf16x2(pr[0], pr[1]));
+        const uint32_t pb1 = transpose8x8_b16(pack_bf16x2(pr[2], pr[3]));
 #pragma unroll
-        for (int u = 0; u < kDecBatch; ++u) {
-            float vf[8];
-            unpack8(vr[u], vf);
-#pragma unroll
-            for (int h = 0; h < G; ++h)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[h][e] = fmaf(pw[h][u], vf[e], acc[h][e]);
+        for (int mt = 0; mt < 8; ++mt) {
+            o[mt][0] *= corr[0]; o[mt][1] *= corr[1]; o[mt][2] *= corr[0]; o[mt][3] *= corr[1];
+            const int w = mt >> 1;
+            const uint32_t sel = (mt & 1) ? 0x7632u : 0x5410u;     // the high / low halves of two rows' words
+            const uint32_t a0 = __byte_perm(word_of(vr[0][0], w), word_of(vr[1][0], w), sel);   // dim 16g + mt,     keys 2t, 2t+1
+            const uint32_t a1 = __byte_perm(word_of(vr[0][1], w), word_of(vr[1][1], w), sel);   // dim 16g + 8 + mt, keys 2t, 2t+1
+            const uint32_t a2 = __byte_perm(word_of(vr[2][0], w), word_of(vr[3][0], w), sel);   // dim 16g + mt,     keys 2t+8, 2t+9
+            const uint32_t a3 = __byte_perm(word_of(vr[2][1], w), word_of(vr[3][1], w), sel);
+            mma_bf16_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
         }
     }
-    // ---- merge: the two half-warps of a warp by shuffle, the 8 warps through shared memory ---------------
+    // ---- the lane's share of l -> the sum over the 8 lanes of equal t; then everything into shared memory ---------
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-        const float mo = __shfl_xor_sync(0xffffffffu, m[h], 16), lo = __shfl_xor_sync(0xffffffffu, l[h], 16);
-        const float mm = fmaxf(m[h], mo);
-        const float c_me = exp2f(m[h] - mm), c_ot = exp2f(mo - mm);
-        l[h] = l[h] * c_me + lo * c_ot;
+    for (int c = 0; c < 2; ++c) {
+        l[c] += __shfl_xor_sync(0xffffffffu, l[c], 4);
+        l[c] += __shfl_xor_sync(0xffffffffu, l[c], 8);
+        l[c] += __shfl_xor_sync(0xffffffffu, l[c], 16);
+    }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float ao = __shfl_xor_sync(0xffffffffu, acc[h][e], 16);
-            acc[h][e] = acc[h][e] * c_me + ao * c_ot;
-        }
-        m[h] = mm;
-        if (half == 0) {
+    for (int c = 0; c < 2; ++c) {
+        const int h = 2 * t + c;
+        if (h < G) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) part_s[warp][h][l16 * 8 + e] = acc[h][e];
-            if (l16 == 0) { part_s[warp][h][kHeadDim] = m[h]; part_s[warp][h][kHeadDim + 1] = l[h]; }
+            for (int mt = 0; mt < 8; ++mt) {
+                part_s[warp][h][16 * g + mt] = o[mt][c];
+                part_s[warp][h][16 * g + 8 + mt] = o[mt][c + 2];
+            }
+            if (g == 0) { part_s[warp][h][kHeadDim] = m[c]; part_s[warp][h][kHeadDim + 1] = l[c]; }
         }
     }
     __syncthreads();
@@ -358,19 +369,19 @@ __global__ void __launch_bounds__(256) decode_attention_gqa_kernel(const DecGqaP
         float M = -1e30f;
 #pragma unroll
         for (int w2 = 0; w2 < 8; ++w2) M = fmaxf(M, part_s[w2][h][kHeadDim]);
-        float L = 0.f, o = 0.f;
+        float L = 0.f, acc = 0.f;
 #pragma unroll
         for (int w2 = 0; w2 < 8; ++w2) {
             const float c = exp2f(part_s[w2][h][kHeadDim] - M);
             L = fmaf(part_s[w2][h][kHeadDim + 1], c, L);
-            o = fmaf(part_s[w2][h][d], c, o);
+            acc = fmaf(part_s[w2][h][d], c, acc);
         }
         const int qh = kh * G + h;
         if (p.n_splits == 1) {
-            p.O[(long long)b * p.o_b + (long long)qh * p.o_h + d] = __float2bfloat16_rn(o / L);
+            p.O[(long long)b * p.o_b + (long long)qh * p.o_h + d] = __float2bfloat16_rn(acc / L);
         } else {
             float* dst = p.partial + (((size_t)b * p.Hq + qh) * p.n_splits + split) * kPartialFloats;
-            dst[d] = o;
+            dst[d] = acc;
             if (d == 0) { dst[kHeadDim] = M; dst[kHeadDim + 1] = L; }
         }
     }
@@ -436,8 +447,19 @@ cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_p
         int sms = 148;
         { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
         const int max_keys = s.window > 0 ? (s.window < s.seq ? s.window : s.seq) : s.seq;   // pos is device data: size for the worst case
-        int n_splits = (2 * sms + s.batch * s.n_kv_heads - 1) / (s.batch * s.n_kv_heads);
-        n_splits = std::max(1, std::min(n_splits, max_keys / 512));                             // at least 512 keys per split
+        // Number of key splits: two CTAs fit an SM, a wave of CTAs costs (a fixed part worth ~192 keys + its keys), and a
+        // partly filled wave costs as much as a full one; take the split count with the cheapest estimate, at least
+        // 256 keys per split.
+        int n_splits = 1;
+        {
+            const long long groups = (long long)s.batch * s.n_kv_heads, slots = 2ll * sms;
+            long long best = -1;
+            for (int n = 1; n <= std::max(1, max_keys / 256); ++n) {
+                const long long waves = (groups * n + slots - 1) / slots;
+                const long long cost = waves * (192 + (max_keys + n - 1) / n);
+                if (best < 0 || cost < best) { best = cost; n_splits = n; }
+            }
+        }
         const size_t need = (size_t)s.batch * s.n_q_heads * n_splits * kPartialFloats * sizeof(float);
         if (n_splits > 1 && (!ctx->workspace || ctx->workspace_bytes < need)) n_splits = 1;
         gp.n_splits = n_splits;
