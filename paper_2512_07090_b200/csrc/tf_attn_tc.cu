@@ -246,6 +246,22 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         return;
     }
 
+    // The softmax threads read the retained indices of the Q rows they will gather (16 lanes per 256-byte row, the
+    // 8 warps take 16 rows per round) and of their own row now, next to the loads the set-up below waits for anyway:
+    // one global round trip less between the set-up and the first Q K^T.
+    constexpr int kRounds = C::kRows / 16;
+    int tq[kRounds];
+    int t_row = -1;
+    if (warp < kMmaWarp) {
+#pragma unroll
+        for (int it = 0; it < kRounds; ++it) {
+            const int s_q = slot0 + it * 16 + warp * 2 + (lane >> 4);
+            tq[it] = s_q < nk ? kept[s_q] : -1;
+        }
+        const int slot_pre = slot0 + (kSplit ? 0 : (warp >> 2) * kTileM) + (tid & (kTileM - 1));
+        if (slot_pre < nk) t_row = kept[slot_pre];
+    }
+
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar_q = sbase + kOffBar;              // Q tiles written
@@ -408,8 +424,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         const int i = warp >> 2;                 // group: its Q tile (shared) or its half of the K/V tiles (split)
         const int r = tid & (kTileM - 1);        // row within the tile
         const int slot = slot0 + (kSplit ? 0 : i * kTileM) + r;
-        const bool valid = slot < nk;
-        const int t_row = valid ? kept[slot] : -1;
+        const bool valid = slot < nk;               // t_row (fetched above) is the row's token position, -1 if none
         int hi = t_row;                                                           // visible keys: lo .. hi
         int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
         if (p.compact && valid) {
@@ -417,16 +432,8 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             hi = slot;
         }
         {
-            // gather the CTA's Q rows into the swizzled K-major operand layout: 16 lanes fetch one row
-            // (256 contiguous bytes), the 8 warps take 16 rows per round
-            constexpr int kRounds = C::kRows / 16;
+            // gather the CTA's Q rows into the swizzled K-major operand layout
             const int sub = lane >> 4, cc = lane & 15, w8 = tid >> 5;
-            int tq[kRounds];
-#pragma unroll
-            for (int it = 0; it < kRounds; ++it) {
-                const int s_q = slot0 + it * 16 + w8 * 2 + sub;
-                tq[it] = s_q < nk ? kept[s_q] : -1;
-            }
             uint4 qv[kRounds];
             const __nv_bfloat16* qbase = p.Q + (long long)b * p.qs.b + (long long)qh * p.qs.h + cc * 8;
 #pragma unroll
