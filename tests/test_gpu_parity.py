@@ -39,6 +39,22 @@ def test_kv_stats_matches_oracle(dtype, B, S, Hkv, scan_path):
     g.close()
 
 
+@pytest.mark.parametrize("scan_path", [1, 2, 3])
+def test_kv_stats_inclusive_mean_every_path(scan_path):
+    """The inclusive-mean anchor (the token itself counted in) on each of the three scan kernels, on a length that
+    leaves a ragged last tile and gives the persistent kernel several tiles per worker on a small grid."""
+    q, k, v = _qkv(3, 1111, 5, 5, torch.bfloat16, seed=21)
+    g = Gpu(q, k, v, anchor_mode=tfb.TF_ANCHOR_INCL_MEAN)
+    g.ctx.tf_set_scan_path(scan_path)
+    for _ in range(2):      # twice: the second launch finds the first one's records and tickets in the scratch
+        g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    g.status_ok()
+    _, kn, vn = oracle_inputs(q, k, v)
+    assert np.abs(to_np(g.sim_k) - oracle.anchor_similarity(kn, tfb.TF_ANCHOR_INCL_MEAN, 0.9)).max() < SCORE_ATOL
+    assert np.abs(to_np(g.sim_v) - oracle.anchor_similarity(vn, tfb.TF_ANCHOR_INCL_MEAN, 0.9)).max() < SCORE_ATOL
+    g.close()
+
+
 @pytest.mark.parametrize("mode,gamma", [(tfb.TF_ANCHOR_INCL_MEAN, 0.9), (tfb.TF_ANCHOR_EMA, 0.9),
                                         (tfb.TF_ANCHOR_EMA, 0.8), (tfb.TF_ANCHOR_EMA, 0.95)])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
@@ -53,15 +69,18 @@ def test_kv_stats_anchor_modes(mode, gamma, dtype):
     g.close()
 
 
-def test_kv_stats_head_major_layout_and_carry():
+@pytest.mark.parametrize("scan_path", [0, 1, 2, 3])
+def test_kv_stats_head_major_layout_and_carry(scan_path):
     """Same values stored [B,H,S,d] (strided view) give the same similarities; two half-sequence
-    calls chained through the carry equal one call; the exported sums are the column sums."""
+    calls chained through the carry equal one call; the exported sums are the column sums.
+    Every scan kernel (plain, Gram one tile per CTA, Gram persistent) takes the same route."""
     B, S, H = 2, 300, 4
     q, k, v = _qkv(B, S, H, H, torch.bfloat16, seed=9)
     kt = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     vt = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     assert kt.stride() != k.stride()
     g = Gpu(q, kt, vt)
+    g.ctx.tf_set_scan_path(scan_path)
     g.ctx.tf_kv_stats(g.shape, g.params, kt, vt, g.sim_k, g.sim_v)
     _, kn, vn = oracle_inputs(q, k, v)
     ref_k, sum_k = oracle.anchor_similarity(kn, want_sum_out=True)
@@ -70,11 +89,13 @@ def test_kv_stats_head_major_layout_and_carry():
     # chained halves
     h = S // 2
     g1 = Gpu(q[:, :h], k[:, :h], v[:, :h])
+    g1.ctx.tf_set_scan_path(scan_path)
     sk = torch.empty(B, H, 128, device=DEV); sv = torch.empty(B, H, 128, device=DEV)
     c1 = tfb.tf_carry(None, None, None, sk.data_ptr(), sv.data_ptr())
     g1.ctx.tf_kv_stats(g1.shape, g1.params, k[:, :h], v[:, :h], g1.sim_k, g1.sim_v, c1)
     cnt = torch.full((B,), h, dtype=torch.int64, device=DEV)
     g2 = Gpu(q[:, h:], k[:, h:], v[:, h:])
+    g2.ctx.tf_set_scan_path(scan_path)
     sk2 = torch.empty_like(sk); sv2 = torch.empty_like(sv)
     c2 = tfb.tf_carry(sk.data_ptr(), sv.data_ptr(), cnt.data_ptr(), sk2.data_ptr(), sv2.data_ptr())
     g2.ctx.tf_kv_stats(g2.shape, g2.params, k[:, h:], v[:, h:], g2.sim_k, g2.sim_v, c2)
