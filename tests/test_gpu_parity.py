@@ -42,7 +42,7 @@ def test_kv_stats_matches_oracle(dtype, B, S, Hkv, scan_path):
 @pytest.mark.parametrize("scan_path", [1, 2, 3])
 def test_kv_stats_inclusive_mean_every_path(scan_path):
     """The inclusive-mean anchor (the token itself counted in) on each of the three scan kernels, on a length that
-    leaves a ragged last tile and gives the persistent kernel several tiles per worker on a small grid."""
+    leaves a ragged last tile."""
     q, k, v = _qkv(3, 1111, 5, 5, torch.bfloat16, seed=21)
     g = Gpu(q, k, v, anchor_mode=tfb.TF_ANCHOR_INCL_MEAN)
     g.ctx.tf_set_scan_path(scan_path)
@@ -52,6 +52,23 @@ def test_kv_stats_inclusive_mean_every_path(scan_path):
     _, kn, vn = oracle_inputs(q, k, v)
     assert np.abs(to_np(g.sim_k) - oracle.anchor_similarity(kn, tfb.TF_ANCHOR_INCL_MEAN, 0.9)).max() < SCORE_ATOL
     assert np.abs(to_np(g.sim_v) - oracle.anchor_similarity(vn, tfb.TF_ANCHOR_INCL_MEAN, 0.9)).max() < SCORE_ATOL
+    g.close()
+
+
+def test_kv_stats_persistent_many_tiles_per_worker():
+    """2048 (tile, tensor) pairs on 888 workers: every worker of the persistent kernel runs its loop more than once
+    (ticket prefetch, barrier phases and TMEM columns carried from tile to tile), and the one-tile kernel must agree."""
+    q, k, v = _qkv(2, 4096, 16, 16, torch.bfloat16, seed=33)
+    g = Gpu(q, k, v)
+    _, kn, vn = oracle_inputs(q, k, v)
+    ref_k, ref_v = oracle.anchor_similarity(kn), oracle.anchor_similarity(vn)
+    for path in (3, 2, 3):
+        g.sim_k.fill_(7.0); g.sim_v.fill_(7.0)
+        g.ctx.tf_set_scan_path(path)
+        g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+        g.status_ok()
+        assert np.abs(to_np(g.sim_k) - ref_k).max() < SCORE_ATOL
+        assert np.abs(to_np(g.sim_v) - ref_v).max() < SCORE_ATOL
     g.close()
 
 
