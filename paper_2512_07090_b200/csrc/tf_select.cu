@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     __shared__ int hist[256];
     __shared__ int s_warp[kSelWarps];
     __shared__ unsigned int s_prefix;
-    __shared__ int s_rank, s_count;
+    __shared__ int s_rank, s_count, s_few_eq;
+    __shared__ unsigned int s_few[32];
 
     grid_dependency_wait();
     const int b = blockIdx.x, tid = threadIdx.x, S = p.S;
@@ -172,6 +173,46 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
                 n_eq = s_count;
                 mask |= 255u << shift;
                 __syncthreads();
+                // Few candidates left under this prefix (typical after two passes: scores share their exponent): one
+                // warp ranks them directly instead of two more histogram passes.  Same result: the key of rank r among
+                // them, how many candidates carry it, and the rank within those.
+                if (shift > 0 && n_eq <= 32) {
+                    if (tid == 0) s_count = 0;
+                    __syncthreads();
+#pragma unroll
+                    for (int i = 0; i < (KPT > 0 ? kChunks : 1 << 30); ++i) {
+                        const int t0 = i * kSelThreads;
+                        if (KPT == 0 && t0 >= S) break;
+                        const int t = t0 + tid;
+                        if (t < S) {
+                            const float sv = score_at(i, t);
+                            if (candidate(t, sv)) {
+                                const unsigned int k = score_key(sv);
+                                if ((k & mask) == prefix) s_few[atomicAdd(&s_count, 1)] = k;
+                            }
+                        }
+                    }
+                    __syncthreads();
+                    if (tid < 32) {
+                        const unsigned int key = tid < n_eq ? s_few[tid] : 0u;
+                        int greater = 0, equal = 0;
+                        for (int o = 0; o < n_eq; ++o) {
+                            const unsigned int ko = __shfl_sync(0xffffffffu, key, o);
+                            greater += ko > key ? 1 : 0;
+                            equal += ko == key ? 1 : 0;
+                        }
+                        if (tid < n_eq && greater < r && r <= greater + equal) {   // every lane holding that key writes the same
+                            s_prefix = key;
+                            s_rank = r - greater;
+                            s_few_eq = equal;
+                        }
+                    }
+                    __syncthreads();
+                    prefix = s_prefix;
+                    r = s_rank;
+                    n_eq = s_few_eq;
+                    break;
+                }
             }
             key_thr = prefix;
             take_eq = r;   // 1 <= r <= n_eq
