@@ -227,7 +227,8 @@ def run_decode(args, wl, tfb, dev, local):
                       "config": workload_config(wl, args), "gpu_launches": int(ctx.launches - launches0),
                       "roofline": {"kernel": "decode_attention", "bound": "hbm", "achieved": cache_bytes / (ms * 1e-3) / 1e9,
                                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": cache_bytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                                   "traffic": None, "peak_kind": pk_kind, "algorithmic_per_launch": cache_bytes}}))
+                                   "traffic": {"c5": 134302464 + 602112}.get(wl.name),   # ncu, profiles/decode_step_c5.txt
+                                   "peak_kind": pk_kind, "algorithmic_per_launch": cache_bytes}}))
     ctx.close()
 
 

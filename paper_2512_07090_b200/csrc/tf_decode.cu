@@ -48,6 +48,10 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_decide_kernel(const Dec
     const bool ema = p.anchor_mode == TF_ANCHOR_EMA, incl = p.anchor_mode == TF_ANCHOR_INCL_MEAN;
     const float a = ema ? p.gamma : 1.f, w = ema ? 1.f - p.gamma : 1.f;
     const long long n_cmp = n0 + (incl ? 1 : 0);            // tokens the anchor covers when it is compared
+    // the controller's state is read now, under the row loads below, not after the block barrier
+    long long steps = 0, skips = 0;
+    float tau_old = 0.f;
+    if (threadIdx.x == 0) { steps = p.steps[b]; skips = p.skips[b]; tau_old = p.tau[b]; }
 
     for (int h = warp; h < p.Hkv; h += kDecWarps) {
         const T* kp = reinterpret_cast<const T*>(p.K) + (long long)b * p.ks.b + (long long)t * p.ks.t + (long long)h * p.ks.h + lane * 4;
@@ -105,11 +109,10 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_decide_kernel(const Dec
             }
             float s = alpha * mk + (1.f - alpha) * mv;
             s += 0.f;
-            const long long steps = p.steps[b], skips = p.skips[b];
             // ratio and step in double, the threshold itself is an fp32 state word
             const double rho = steps > 0 ? (double)skips / (double)steps : 0.0;
             const double delta = (double)p.eta * (p.alg1_sign ? ((double)p.target - rho) : (rho - (double)p.target));
-            const float tau = p.tau[b] + (float)delta;
+            const float tau = tau_old + (float)delta;
             const bool decide = s > tau;              // false for NaN
             const bool skip = decide && t >= p.warmup;
             p.tau[b] = tau;
@@ -464,6 +467,9 @@ cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_p
         if (n_splits > 1 && (!ctx->workspace || ctx->workspace_bytes < need)) n_splits = 1;
         gp.n_splits = n_splits;
         gp.partial = n_splits > 1 ? static_cast<float*>(ctx->workspace) : nullptr;
+        // the partial results overwrite the start of the workspace, where tf_kv_stats keeps its tagged records: the
+        // next scan on this workspace clears its region first instead of trusting what it finds there
+        if (n_splits > 1) { ctx->scan_user.needs_clear = true; ctx->scan_owned.needs_clear = true; }
         const dim3 grid((unsigned)n_splits, (unsigned)s.n_kv_heads, (unsigned)s.batch);
         switch (G) {
             case 1: e = launch_dependent(decode_attention_gqa_kernel<1>, grid, dim3(256), 0, st, gp); break;

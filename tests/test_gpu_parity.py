@@ -329,6 +329,46 @@ def test_layer_filter_host_entry_matches_device_entry():
     g.close()
 
 
+def test_decode_and_prefill_share_the_workspace():
+    """The decode step keeps its split-key partial results in the bound workspace, over the region where the
+    similarity scan keeps its records; a scan after decode steps must still be right (it clears its region first),
+    and the split decode output must equal the one-CTA-per-head output computed without a workspace."""
+    B, S, Hq, Hkv = 2, 2304, 8, 2
+    q, k, v = _qkv(B, S, Hq, Hkv, torch.bfloat16, seed=77)
+    _, kn, vn = oracle_inputs(q, k, v)
+    ref_k = oracle.anchor_similarity(kn)
+    ctx = tfb.Context(0)
+    params = tfb.default_params(prune_ratio=0.25, warmup_tokens=4)
+    pshape = tfb.make_shape(None, k, v)
+    ctx.ensure_workspace(pshape, params)
+    sk = torch.empty(B, S, Hkv, device=DEV); sv = torch.empty_like(sk)
+    shape = tfb.make_shape(None, k, v, n_q_heads=Hq)
+    O = torch.empty(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    shape.q_stride[:] = [q.stride(0), 0, q.stride(2)]
+    shape.o_stride[:] = [O.stride(0), 0, O.stride(1)]
+    score = torch.empty(B, device=DEV); skip = torch.empty(B, dtype=torch.uint8, device=DEV)
+    pos = torch.full((B,), S - 1, dtype=torch.int32, device=DEV)
+    outs = []
+    for rnd in range(2):
+        ctx.tf_kv_stats(pshape, params, k, v, sk, sv)
+        assert np.abs(to_np(sk) - ref_k).max() < SCORE_ATOL, rnd
+        st = tfb.DecodeState(B, Hkv, DEV, tau0=10.0)          # a threshold no score reaches: attention always runs
+        n0 = ctx.launches
+        ctx.tf_decode_step(shape, params, 0.0, q[:, S - 1], k, v, pos, st, O, score, skip)
+        assert ctx.launches - n0 == 3                          # decide, split attention, combine
+        outs.append(O.clone())
+    ctx.set_workspace(None)
+    st = tfb.DecodeState(B, Hkv, DEV, tau0=10.0)
+    n0 = ctx.launches
+    ctx.tf_decode_step(shape, params, 0.0, q[:, S - 1], k, v, pos, st, O, score, skip)
+    assert ctx.launches - n0 == 2                              # no workspace: one CTA per KV head, no combine
+    code, det = ctx.tf_get_status()
+    assert code == tfb.TF_OK, det
+    assert torch.equal(outs[0], outs[1])
+    assert attn_rel_err(to_np(outs[0]), to_np(O)) < 1e-2       # same products, different split of the softmax sums
+    ctx.close()
+
+
 def test_device_rejects_bad_arguments_without_launching():
     q, k, v = _qkv(1, 64, 2, 2, torch.bfloat16)
     g = Gpu(q, k, v)
