@@ -698,7 +698,8 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     } else if (!make_kv_map(&mapK, K, s.k_stride, s.batch, s.seq, s.n_kv_heads) ||
                !make_kv_map(&mapV, V, s.v_stride, s.batch, s.seq, s.n_kv_heads))
         return cudaErrorNotSupported;
-    static bool attr_set = false;
+    static bool attr_set_dev[kDeviceFlagSlots] = {};      // function attributes are per device
+    bool& attr_set = attr_set_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg<false>::kSmemBytes);

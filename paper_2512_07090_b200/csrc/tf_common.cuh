@@ -10,6 +10,7 @@
 namespace tf {
 
 constexpr int kHeadDim = 128;
+constexpr int kDeviceFlagSlots = 64;       // per-device one-time set-up flags
 constexpr float kNormEps = 1e-8f;   // lower clamp of each norm in the cosine
 
 // Device status record: four 64-bit words {code, where, nan_count, reserved}.

@@ -719,7 +719,8 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
         !make_bshd_map(&mv, V, s.v_stride, s.batch, s.seq, s.n_kv_heads, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kGT,
                        CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorNotSupported;
-    static bool attr_set = false;
+    static bool attr_set_dev[kDeviceFlagSlots] = {};      // function attributes are per device
+    bool& attr_set = attr_set_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kv_stats_gram1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kT1Smem);
         if (e != cudaSuccess) return e;
@@ -748,7 +749,8 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     // cross-over between 2.3 and 11.5 tiles per worker); below that the one-tile-per-CTA form starts sooner
     const bool persistent = ctx->scan_path == 3 || (ctx->scan_path == 0 && 2 * tiles >= (size_t)4 * sms * kPWorkers);
     if (persistent) {
-        static bool attr_set_p = false;
+        static bool attr_set_p_dev[kDeviceFlagSlots] = {};
+        bool& attr_set_p = attr_set_p_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
         if (!attr_set_p) {
             cudaError_t e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
             if (e != cudaSuccess) return e;
