@@ -57,6 +57,7 @@ struct TcParams {
     int compact;          // 1: K / V hold the retained tokens only, entry c = token kept_idx[c] (TF_KV_RETAINED)
     int n_row_blocks;     // CTAs per (batch, query head)
     int heads_fastest;    // CTA order: 1 = all heads of the heaviest row block first, 0 = all row blocks of a head together
+    int first_pair;       // row block the first CTA of a head takes: the last one expected to hold retained rows
 };
 
 // Two ways of giving the two softmax groups of a CTA their work:
@@ -231,7 +232,11 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     const int n_bh = (int)(gridDim.x / (unsigned)p.n_row_blocks);
     const int rb = p.heads_fastest ? (int)blockIdx.x / n_bh : (int)blockIdx.x % p.n_row_blocks;
     const int bh = p.heads_fastest ? (int)blockIdx.x % n_bh : (int)blockIdx.x / p.n_row_blocks;
-    const int pair = p.n_row_blocks - 1 - rb;
+    // Row blocks are taken from the heaviest expected one (the last with retained rows, a host-side estimate) down to
+    // block 0, then the blocks above the estimate, which are normally empty: CTAs with nothing to do start last
+    // instead of delaying the first wave of real work.  Any estimate gives a one-to-one assignment.
+    int pair = p.first_pair - rb;
+    if (pair < 0) pair += p.n_row_blocks;
     const int qh = bh % p.Hq, b = bh / p.Hq;
     const int nk = p.n_kept[b];
     const int slot0 = pair * C::kRows;
@@ -738,6 +743,12 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 1.0 * sms);
     const int rows_per_cta = split ? kTileM : kQTiles * kTileM;
     tp.n_row_blocks = (s.seq + rows_per_cta - 1) / rows_per_cta;
+    {
+        const long long kept_est = (p.select_mode == TF_SELECT_RATIO) ? (long long)s.seq - (long long)floor(p.prune_ratio * (double)s.seq)
+                                                                      : (long long)s.seq;
+        const long long blocks = (std::max<long long>(kept_est, 1) + rows_per_cta - 1) / rows_per_cta;
+        tp.first_pair = (int)std::min<long long>(std::max<long long>(blocks - 1, 0), tp.n_row_blocks - 1);
+    }
     const double kv_bytes = 2.0 * s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
     tp.heads_fastest = (kv_bytes <= 48e6 || ctas_shared < 6.0 * sms) ? 1 : 0;   // K and V stay in L2, or balance matters more
     const long long n_ctas = (long long)tp.n_row_blocks * s.n_q_heads * s.batch;
