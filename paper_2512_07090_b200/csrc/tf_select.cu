@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     __shared__ int hist[256];
     __shared__ int s_warp[kSelWarps];
     __shared__ unsigned int s_prefix;
-    __shared__ int s_rank, s_count, s_few_eq;
+    __shared__ int s_rank, s_count, s_few_eq, s_total;
+    __shared__ int s_tab[KPT > 0 ? KPT : 1][kSelWarps];   // [chunk][warp] ballot counts of the final sweep
     __shared__ unsigned int s_few[32];
 
     grid_dependency_wait();
@@ -222,34 +223,115 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     // ---- sweep in index order: decide, count equals, compact ---------------------------------------
     int kept_base = 0, eq_base = 0;
     float th_min = CUDART_INF_F;
+    if constexpr (KPT > 0) {
+        // Register form: ranks in index order (token = chunk * 1024 + thread) come from ONE block-wide scan of a
+        // [chunk][warp] table of ballot counts per question (rank among the equal keys, position among the kept
+        // tokens), instead of two block scans per chunk of 1024 tokens.
+        int* tab = &s_tab[0][0];
+        const int lane = tid & 31, wid = tid >> 5;
+        const unsigned int lt = (1u << lane) - 1u;
+        auto scan_table = [&]() {          // exclusive prefix over tab[0 .. KPT*32), in place; s_total = the sum
+            __syncthreads();
+            if (wid == 0) {
+                int v[NR], sum = 0;
 #pragma unroll
-    for (int i = 0; i < (KPT > 0 ? kChunks : 1 << 30); ++i) {
-        const int t0 = i * kSelThreads;
-        if (t0 >= S) break;
-        const int t = t0 + tid;
-        const bool in = t < S;
-        const float s = in ? score_at(i, t) : 0.f;
-        const bool cand = in && candidate(t, s);
-        bool prune = false;
-        if (p.mode == TF_SELECT_THRESHOLD) {
-            prune = cand && (s > tau);
-        } else if (!nothing) {
-            const unsigned int k = cand ? score_key(s) : 0u;
-            const bool eq = cand && (k == key_thr);
-            int eq_tot;
-            const int eq_rank = block_rank(eq, s_warp, eq_tot) + eq_base;   // 0-based among equals
-            eq_base += eq_tot;
-            // the take_eq equals with the highest index: ranks n_eq-take_eq .. n_eq-1
-            prune = cand && ((k > key_thr) || (eq && eq_rank >= n_eq - take_eq));
+                for (int e = 0; e < NR; ++e) { v[e] = tab[lane * NR + e]; sum += v[e]; }
+                int incl = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += n;
+                }
+                int run = incl - sum;
+#pragma unroll
+                for (int e = 0; e < NR; ++e) { tab[lane * NR + e] = run; run += v[e]; }
+                if (lane == 31) s_total = incl;
+            }
+            __syncthreads();
+        };
+        unsigned int eq_bits = 0, prune_bits = 0;
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int t = i * kSelThreads + tid;
+            const float sv = sreg[i];
+            const bool cand = t < S && candidate(t, sv);
+            if (p.mode == TF_SELECT_THRESHOLD) {
+                if (cand && sv > tau) prune_bits |= 1u << i;
+            } else if (!nothing && cand) {
+                const unsigned int k = score_key(sv);
+                if (k > key_thr) prune_bits |= 1u << i;
+                if (k == key_thr) eq_bits |= 1u << i;
+            }
         }
-        if (prune) th_min = fminf(th_min, s);
-        const bool keep = in && !prune;
-        int kept_tot;
-        const int pos = block_rank(keep, s_warp, kept_tot) + kept_base;
-        kept_base += kept_tot;
-        if (in) {
-            p.keep_mask[(size_t)b * S + t] = keep ? 1 : 0;
-            if (keep) p.kept_idx[(size_t)b * S + pos] = t;
+        if (p.mode != TF_SELECT_THRESHOLD && !nothing) {      // CTA-uniform
+#pragma unroll
+            for (int i = 0; i < NR; ++i) {
+                const unsigned int bal = __ballot_sync(0xffffffffu, (eq_bits >> i) & 1u);
+                if (lane == 0) tab[i * kSelWarps + wid] = __popc(bal);
+            }
+            scan_table();
+#pragma unroll
+            for (int i = 0; i < NR; ++i) {
+                const bool eq = (eq_bits >> i) & 1u;
+                const unsigned int bal = __ballot_sync(0xffffffffu, eq);
+                const int eq_rank = tab[i * kSelWarps + wid] + __popc(bal & lt);     // 0-based among equals, index order
+                // the take_eq equals with the highest index: ranks n_eq-take_eq .. n_eq-1
+                if (eq && eq_rank >= n_eq - take_eq) prune_bits |= 1u << i;
+            }
+            __syncthreads();                                   // the table is reused below
+        }
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int t = i * kSelThreads + tid;
+            const bool keep = t < S && !((prune_bits >> i) & 1u);
+            const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) tab[i * kSelWarps + wid] = __popc(bal);
+        }
+        scan_table();
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int t = i * kSelThreads + tid;
+            const bool in = t < S, prune = (prune_bits >> i) & 1u;
+            const bool keep = in && !prune;
+            const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+            const int pos = tab[i * kSelWarps + wid] + __popc(bal & lt);
+            if (prune) th_min = fminf(th_min, sreg[i]);
+            if (in) {
+                p.keep_mask[(size_t)b * S + t] = keep ? 1 : 0;
+                if (keep) p.kept_idx[(size_t)b * S + pos] = t;
+            }
+        }
+        kept_base = s_total;
+    } else {
+    #pragma unroll
+        for (int i = 0; i < (KPT > 0 ? kChunks : 1 << 30); ++i) {
+            const int t0 = i * kSelThreads;
+            if (t0 >= S) break;
+            const int t = t0 + tid;
+            const bool in = t < S;
+            const float s = in ? score_at(i, t) : 0.f;
+            const bool cand = in && candidate(t, s);
+            bool prune = false;
+            if (p.mode == TF_SELECT_THRESHOLD) {
+                prune = cand && (s > tau);
+            } else if (!nothing) {
+                const unsigned int k = cand ? score_key(s) : 0u;
+                const bool eq = cand && (k == key_thr);
+                int eq_tot;
+                const int eq_rank = block_rank(eq, s_warp, eq_tot) + eq_base;   // 0-based among equals
+                eq_base += eq_tot;
+                // the take_eq equals with the highest index: ranks n_eq-take_eq .. n_eq-1
+                prune = cand && ((k > key_thr) || (eq && eq_rank >= n_eq - take_eq));
+            }
+            if (prune) th_min = fminf(th_min, s);
+            const bool keep = in && !prune;
+            int kept_tot;
+            const int pos = block_rank(keep, s_warp, kept_tot) + kept_base;
+            kept_base += kept_tot;
+            if (in) {
+                p.keep_mask[(size_t)b * S + t] = keep ? 1 : 0;
+                if (keep) p.kept_idx[(size_t)b * S + pos] = t;
+            }
         }
     }
     for (int i = kept_base + tid; i < S; i += kSelThreads) p.kept_idx[(size_t)b * S + i] = -1;
