@@ -99,6 +99,10 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel on the stream (if launched with launch_dependent) become resident now instead of when this
+// grid has exited; its grid_dependency_wait() still waits for this grid to complete.  For small grids only: the
+// waiting CTAs of the next kernel occupy SM resources.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 }  // namespace tf
 

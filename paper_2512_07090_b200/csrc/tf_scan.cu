@@ -368,6 +368,7 @@ __global__ void __launch_bounds__(256) score_fuse_kernel(const float* __restrict
                                                          const float* __restrict__ sim_v,
                                                          float* __restrict__ score, long long n_tokens,
                                                          int H, int mode, float eps, DevStatus* status) {
+    grid_launch_dependents();   // a short kernel: the selection CTAs may become resident while it runs
     grid_dependency_wait();
     const long long tok = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;

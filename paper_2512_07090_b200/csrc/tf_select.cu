@@ -68,6 +68,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     __shared__ int s_tab[KPT > 0 ? KPT : 1][kSelWarps];   // [chunk][warp] ballot counts of the final sweep
     __shared__ unsigned int s_few[32];
 
+    grid_launch_dependents();   // one CTA per sequence: the attention grid may take the other SMs and set up meanwhile
     grid_dependency_wait();
     const int b = blockIdx.x, tid = threadIdx.x, S = p.S;
     const float* sc = p.score + (size_t)b * S;
