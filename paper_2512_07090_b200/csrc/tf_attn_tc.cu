@@ -225,6 +225,29 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     constexpr int kStages = C::kStages, kOffQ = C::kOffQ, kOffRing = C::kOffRing, kOffBar = C::kOffBar, kStep = C::kStep;
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_q = sbase + kOffBar;              // Q tiles written
+    const uint32_t bar_full = bar_q + 8;                 // [kStages] ring slot filled by TMA
+    const uint32_t bar_empty = bar_full + 8 * kStages;   // [kStages] ring slot consumed by the MMAs
+    const uint32_t bar_s = bar_empty + 8 * kStages;      // [2] S_i ready
+    const uint32_t bar_p = bar_s + 16;                   // [2] P_i written (and O_i rescaled)
+    const uint32_t bar_o = bar_p + 16;                   // all MMAs done
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 160);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar + 168);
+    // Barriers and TMEM need nothing from global memory: they are set up before the wait for the previous kernel,
+    // which (the selection, one CTA per sequence) lets this grid become resident while it still runs.  Every way
+    // out of the kernel from here on gives the TMEM columns back.
+    if (tid == 0) {
+        mbar_init(bar_q, kSoftmaxThreads);
+        for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, kTileM); }
+        mbar_init(bar_o, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     grid_dependency_wait();   // kept_idx / n_kept come from the kernel before this one
     // CTAs start in index order.  Row blocks of a head differ in length by the causal triangle, so the
     // heaviest go first; with few CTAs per SM that has to hold across heads (heads_fastest), while a
@@ -240,14 +263,18 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     const int qh = bh % p.Hq, b = bh / p.Hq;
     const int nk = p.n_kept[b];
     const int slot0 = pair * C::kRows;
-    if (slot0 >= max(nk, 1)) return;
-
     const int32_t* kept = p.kept_idx + (size_t)b * p.S;
     __nv_bfloat16* Ob = p.O + (long long)b * p.os.b + (long long)qh * p.os.h;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
-    if (nk == 0) {   // nothing retained: the whole head is zero
-        for (int i = tid; i < p.S * 16; i += kThreads)
-            *reinterpret_cast<uint4*>(Ob + (long long)(i >> 4) * p.os.t + (i & 15) * 8) = zero4;
+    if (slot0 >= max(nk, 1) || nk == 0) {   // no retained row in this block (CTA-uniform)
+        if (slot0 < max(nk, 1)) {           // nothing retained at all: the whole head is zero
+            for (int i = tid; i < p.S * 16; i += kThreads)
+                *reinterpret_cast<uint4*>(Ob + (long long)(i >> 4) * p.os.t + (i & 15) * 8) = zero4;
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        if (warp == kMmaWarp) tmem_dealloc(*tmem_slot, kTmemCols);
         return;
     }
 
@@ -266,17 +293,6 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         const int slot_pre = slot0 + (kSplit ? 0 : (warp >> 2) * kTileM) + (tid & (kTileM - 1));
         if (slot_pre < nk) t_row = kept[slot_pre];
     }
-
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar_q = sbase + kOffBar;              // Q tiles written
-    const uint32_t bar_full = bar_q + 8;                 // [kStages] ring slot filled by TMA
-    const uint32_t bar_empty = bar_full + 8 * kStages;   // [kStages] ring slot consumed by the MMAs
-    const uint32_t bar_s = bar_empty + 8 * kStages;      // [2] S_i ready
-    const uint32_t bar_p = bar_s + 16;                   // [2] P_i written (and O_i rescaled)
-    const uint32_t bar_o = bar_p + 16;                   // all MMAs done
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 160);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar + 168);
 
     // ---- which K/V tiles each Q tile needs (CTA-uniform) -------------------------------------------
     // group i works on tiles jb[i], jb[i] + kStep, ... < je[i]
@@ -303,16 +319,6 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     const int J0 = jb[0], J1 = max(je[0], je[1]);   // rows ascend, so tile 0 starts first
     const int kh = qh / (p.Hq / p.Hkv);
 
-    if (tid == 0) {
-        mbar_init(bar_q, kSoftmaxThreads);
-        for (int i = 0; i < kStages; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, kTileM); }
-        mbar_init(bar_o, 1);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncwarp();
-    if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
