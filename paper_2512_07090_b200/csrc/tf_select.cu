@@ -102,28 +102,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     if (p.mode == TF_SELECT_THRESHOLD) {
         tau = p.threshold[b];
     } else {
-        // E = number of candidates
-        int e_local = 0;
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < NR; ++i) { const int t = i * kSelThreads + tid; e_local += (t < S && candidate(t, score_at(i, t))) ? 1 : 0; }
-        } else {
-            for (int t = tid; t < S; t += kSelThreads) e_local += candidate(t, sc[t]) ? 1 : 0;
-        }
-        if (tid == 0) s_count = 0;
-        __syncthreads();
-        e_local = __reduce_add_sync(0xffffffffu, e_local);
-        if ((tid & 31) == 0) atomicAdd(&s_count, e_local);
-        __syncthreads();
-        const long long E = s_count;
-        long long P = p.p_target < E ? p.p_target : E;
-        __syncthreads();
-        if (P <= 0) {
+        if (p.p_target <= 0) {
             nothing = true;
         } else {
-            // radix select: rank r (1-based from the top) among candidates matching the prefix so far
+            // radix select: rank r (1-based from the top) among candidates matching the prefix so far.  The number
+            // of candidates E, which caps the number to prune (P = min(E, target)), is the total of the first pass's
+            // histogram.
             unsigned int prefix = 0, mask = 0;
-            int r = (int)P;
+            int r = 0;
             for (int shift = 24; shift >= 0; shift -= 8) {
                 for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
                 __syncthreads();
@@ -158,6 +144,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
                     if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
                 }
                 __syncthreads();
+                if (shift == 24) {                       // first pass: E is known now (uniform over the CTA)
+                    int E = 0;
+#pragma unroll
+                    for (int w2 = 0; w2 < 8; ++w2) E += s_warp[w2];
+                    r = (int)(p.p_target < (long long)E ? p.p_target : (long long)E);
+                    if (r <= 0) { nothing = true; break; }
+                }
                 if (tid < 256) {
                     int off = 0;
                     for (int w2 = 0; w2 < (tid >> 5); ++w2) off += s_warp[w2];
@@ -174,11 +167,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
                 r = s_rank;
                 n_eq = s_count;
                 mask |= 255u << shift;
-                __syncthreads();
+                // (no barrier here: the next pass writes s_prefix, s_rank and s_count only after two more barriers)
                 // Few candidates left under this prefix (typical after two passes: scores share their exponent): one
                 // warp ranks them directly instead of two more histogram passes.  Same result: the key of rank r among
                 // them, how many candidates carry it, and the rank within those.
                 if (shift > 0 && n_eq <= 32) {
+                    __syncthreads();                          // everybody has read s_count
                     if (tid == 0) s_count = 0;
                     __syncthreads();
 #pragma unroll
