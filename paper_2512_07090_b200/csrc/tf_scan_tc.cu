@@ -31,7 +31,6 @@ constexpr int kHalf = 128 * 128;               // one [128 rows][128 B] swizzled
 constexpr int kXBytes = 2 * kHalf;             // one tensor's tile
 constexpr int kBtBytes = 2 * 16 * 128;         // small B operand: [16 rows][128 elements], two 64-element blocks
 constexpr int kGramAnchorEvery = 4;             // a prefix record every 4th chunk: at most 4 aggregates + 1 prefix per look-back
-constexpr int kGramPollBatch = 4;
 constexpr long long kGramWaitCycles = 1000000000ll;
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------------
@@ -192,8 +191,15 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     const bool has_prev = c > 0;
     const int a0 = has_prev ? ((c - 1) / kGramAnchorEvery) * kGramAnchorEvery : 0;
     const uint2* prec = prefix_rec + ((size_t)(a0 / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid;
-    uint2 pfirst = make_uint2(0, 0);
-    if (has_prev) pfirst = ld_packet2(prec);
+    uint2 pfirst = make_uint2(0, 0), afirst[kGramAnchorEvery];
+    const uint2* arec = agg_rec + ((size_t)a0 * p.n_chains + chain) * kHeadDim + tid;      // chunk a0 + u: u n_chains records on
+    const size_t astride = (size_t)p.n_chains * kHeadDim;
+    if (has_prev) {
+        pfirst = ld_packet2(prec);
+#pragma unroll
+        for (int u = 0; u < kGramAnchorEvery; ++u)
+            if (a0 + u < c) afirst[u] = ld_packet2(arec + u * astride);
+    }
 
     uint32_t mma_phase = 0;
     wait_bar(bar_tma, 0, abort_flag, p.status, 100);
@@ -229,17 +235,9 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
             if (p.sum_in[x]) carry = p.sum_in[x][(size_t)chain * kHeadDim + tid];
         } else {
             float A = 0.f;
-            for (int j0 = a0; j0 < c; j0 += kGramPollBatch) {
-                uint2 r[kGramPollBatch];
 #pragma unroll
-                for (int u = 0; u < kGramPollBatch; ++u)
-                    if (j0 + u < c) r[u] = ld_packet2(agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid);
-#pragma unroll
-                for (int u = 0; u < kGramPollBatch; ++u)
-                    if (j0 + u < c)
-                        A += wait_packet2(agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u], p.epoch,
-                                          p.max_polls, p.status, tile);
-            }
+            for (int u = 0; u < kGramAnchorEvery; ++u)       // requested while the tile was in flight
+                if (a0 + u < c) A += wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile);
             carry = wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile) + A;
         }
         if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
@@ -345,8 +343,14 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
         const long long cnt = (p.count_in ? p.count_in[b] : 0ll) + t_tok + (p.incl ? 1 : 0);
         float cosv = 0.f;
         if (cnt > 0) {
-            const float s = 1.f / (float)cnt;      // anchor = sum * s
-            cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pp, 0.f)) * s, kNormEps));
+            // anchor = sum / cnt; the 1 / cnt cancels unless a norm falls under its clamp
+            const float fc = (float)cnt, lim = kNormEps * kNormEps;
+            if (g_diag > lim && pp > lim * fc * fc) {
+                cosv = d * rsqrtf(g_diag) * rsqrtf(pp);
+            } else {
+                const float s = 1.f / fc;
+                cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pp, 0.f)) * s, kNormEps));
+            }
         }
         p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = cosv;
     }
