@@ -196,6 +196,22 @@ def test_select_bit_exact_ties_eligibility_nan_threshold(case):
         _select_case(coarse, 0.5, 3, elig, tfb.TF_SELECT_THRESHOLD, [5.0, 0.0])  # nothing / a lot
 
 
+@pytest.mark.parametrize("n_tied", [2, 20, 32, 33, 200])
+@pytest.mark.parametrize("S", [1500, 5000, 20000])      # two / eight scores per thread in registers, scores re-read
+def test_select_few_candidates_left_with_ties_at_the_cut(S, n_tied):
+    """The cut falls inside a group of exactly equal scores among otherwise distinct ones: after a pass or two
+    the radix select has few candidates left under its prefix (one warp ranks them when there are at most 32),
+    some of them tied, and the ties must go highest index first, exactly as the oracle takes them."""
+    rng = np.random.default_rng(S + n_tied)
+    score = rng.normal(0.2, 0.2, (2, S)).astype(np.float32)
+    P = int(np.floor(0.5 * S))
+    for b in range(2):
+        order = np.argsort(-score[b], kind="stable")
+        cut = order[P - n_tied // 2: P - n_tied // 2 + n_tied]     # the scores around rank P
+        score[b, cut] = score[b, order[P]]
+    _select_case(score, 0.5, warm=3)
+
+
 # ------------------------------------------------------------------------------- a5
 # path 2 / 3: the tensor-core kernel with K/V tiles shared by two Q tiles / split between the softmax groups
 @pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 1),
@@ -268,6 +284,25 @@ def test_pruned_attention_nothing_kept_and_everything_kept(path):
     qn, kn, vn = oracle_inputs(q, k, v)
     dense = oracle.pruned_attention(qn, kn, vn, np.ones((2, 70), np.uint8))
     assert attn_rel_err(o[1], dense[1]) < ATTN_TOL[torch.bfloat16]
+    g.close()
+
+
+@pytest.mark.parametrize("tensor_cores", [2, 3])
+@pytest.mark.parametrize("claimed_ratio", [0.0, 0.9])
+def test_pruned_attention_with_a_retained_list_the_ratio_does_not_predict(tensor_cores, claimed_ratio):
+    """tf_pruned_attention takes any retained list; the kernel orders its row blocks by the count the prune ratio
+    suggests.  With a list much longer or much shorter than that, every row block must still be served once."""
+    B, S, Hq, Hkv = 2, 1500, 4, 2
+    q, k, v = _qkv(B, S, Hq, Hkv, torch.bfloat16, seed=5)
+    qn, kn, vn = oracle_inputs(q, k, v)
+    ref = oracle.layer_filter(qn, kn, vn, prune_ratio=0.4, warmup_tokens=1)      # the list really keeps 60 %
+    g = Gpu(q, k, v, prune_ratio=claimed_ratio)
+    g.ctx.tf_set_attention_path(tensor_cores)
+    g.O.fill_(float("nan"))
+    g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, torch.from_numpy(ref["kept_idx"]).to(DEV),
+                              torch.from_numpy(ref["n_kept"]).to(DEV), g.O)
+    g.status_ok()
+    assert attn_rel_err(to_np(g.O), ref["O"]) < ATTN_TOL[torch.bfloat16]
     g.close()
 
 
