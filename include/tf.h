@@ -178,8 +178,12 @@ tf_status tf_layer_filter(tf_ctx *ctx, const tf_shape *shape, const tf_filter_pa
 
 /* The same layer step for callers whose tensors live in HOST memory (pinned memory makes the
  * copies asynchronous): copies Q, K, V to device staging buffers that the context owns and grows
- * on demand (this entry point allocates; it also binds its own workspace), runs tf_layer_filter,
- * copies O and the optional outputs back and synchronises the stream before returning.
+ * on demand (this entry point allocates; it also binds its own workspace, and on first use creates two
+ * internal streams), runs the steps of tf_layer_filter, copies O and the optional outputs back and
+ * synchronises before returning.  The copies are pipelined over both directions of the host link:
+ * K and V go first (steps a1-a4 need no Q), then Q arrives in up to eight groups of query heads
+ * (whole KV-head groups, at least 2 MB each) while the attention of the group before runs on the
+ * caller's stream and its output rows travel back.
  * shape strides describe the host tensors; they must be dense token-major [B,S,H,128]. */
 tf_status tf_layer_filter_host(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
                                const void *Q_host, const void *K_host, const void *V_host,

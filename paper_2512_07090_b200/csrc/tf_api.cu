@@ -146,6 +146,11 @@ tf_status tf_destroy(tf_ctx* ctx) {
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     if (ctx->stage) cudaFree(ctx->stage);
     if (ctx->owned_ws) cudaFree(ctx->owned_ws);
+    if (ctx->host_streams_ready) {
+        cudaStreamDestroy(ctx->s_in);
+        cudaStreamDestroy(ctx->s_out);
+        for (int i = 0; i < tf_ctx::kHostEvents; ++i) cudaEventDestroy(ctx->ev[i]);
+    }
     delete ctx;
     return TF_OK;
 }
@@ -303,27 +308,88 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         ctx->scan_owned.ptr = ctx->owned_ws;
     }
     char* base = static_cast<char*>(ctx->stage);
-    void* dQ = base; void* dO = base + qb; void* dK = base + 2 * qb; void* dV = base + 2 * qb + kb;
+    char* dQ = base; char* dO = base + qb; void* dK = base + 2 * qb; void* dV = base + 2 * qb + kb;
     float* dS = reinterpret_cast<float*>(base + 2 * qb + 2 * kb);
     uint8_t* dM = reinterpret_cast<uint8_t*>(base + 2 * qb + 2 * kb + sb);
     int32_t* dI = reinterpret_cast<int32_t*>(base + 2 * qb + 2 * kb + sb + mb);
     int32_t* dN = reinterpret_cast<int32_t*>(base + 2 * qb + 2 * kb + sb + mb + ib);
-    cudaError_t e = cudaMemcpyAsync(dQ, Q_host, tokens * shape->n_q_heads * d * es, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(dK, K_host, tokens * shape->n_kv_heads * d * es, cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(dV, V_host, tokens * shape->n_kv_heads * d * es, cudaMemcpyHostToDevice, st);
+
+    // Pipeline over the two directions of the host link: K and V go first (the filter needs all of them and no
+    // Q), then Q arrives in groups of query heads while the attention of the group before runs and its output
+    // rows travel back.  Copies in: one internal stream; kernels: the caller's stream; copies out: a second
+    // internal stream; events chain them.
+    if (!ctx->host_streams_ready) {
+        if (cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking) != cudaSuccess)
+            return TF_ERR_CUDA;
+        for (int i = 0; i < tf_ctx::kHostEvents; ++i)
+            if (cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) != cudaSuccess) return TF_ERR_CUDA;
+        ctx->host_streams_ready = true;
+    }
+    const int gqa = shape->n_q_heads / shape->n_kv_heads;
+    int groups = 1;                                           // head groups of whole KV-head groups, >= 2 MB of Q each
+    for (int g2 : {8, 4, 2})
+        if (groups == 1 && shape->n_q_heads % g2 == 0 && (shape->n_q_heads / g2) % gqa == 0 &&
+            tokens * (size_t)(shape->n_q_heads / g2) * d * es >= ((size_t)2 << 20))
+            groups = g2;
+    const int hq_g = shape->n_q_heads / groups, hkv_g = shape->n_kv_heads / groups;
+    cudaEvent_t ev_start = ctx->ev[0], ev_kv = ctx->ev[1], ev_sel = ctx->ev[2];
+    cudaError_t e = cudaEventRecord(ev_start, st);             // whatever the caller queued before is done first
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_in, ev_start, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_out, ev_start, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dK, K_host, tokens * shape->n_kv_heads * d * es, cudaMemcpyHostToDevice, ctx->s_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dV, V_host, tokens * shape->n_kv_heads * d * es, cudaMemcpyHostToDevice, ctx->s_in);
+    if (e == cudaSuccess) e = cudaEventRecord(ev_kv, ctx->s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, ev_kv, 0);
     if (e != cudaSuccess) return TF_ERR_CUDA;
+
     void* saved_ws = ctx->workspace; const size_t saved_bytes = ctx->workspace_bytes;
     ctx->workspace = ctx->owned_ws; ctx->workspace_bytes = ctx->owned_ws_bytes;
-    s = tf_layer_filter(ctx, shape, params, dQ, dK, dV, dO, dS, dM, dI, dN, stream);
+    {   // steps a1-a4 on the device copies (the same launches tf_layer_filter makes)
+        char* ws = static_cast<char*>(ctx->workspace);
+        float* sim_k = reinterpret_cast<float*>(ws + w.sim_k);
+        float* sim_v = reinterpret_cast<float*>(ws + w.sim_v);
+        float* theta = reinterpret_cast<float*>(ws + w.theta);
+        tf_shape ds = *shape;                                  // device copies are dense like the host tensors
+        e = launch_kv_stats(ctx, ds, *params, dK, dV, sim_k, sim_v, nullptr, &ctx->scan_owned, st);
+        if (e == cudaSuccess) e = launch_score_fuse(ctx, ds, *params, sim_k, sim_v, dS, st);
+        if (e == cudaSuccess) e = launch_select(ctx, ds, *params, dS, dM, dI, dN, theta, st);
+        if (e == cudaSuccess) e = cudaEventRecord(ev_sel, st);
+    }
+    s = e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    const size_t row = (size_t)shape->n_q_heads * d * es, row_g = (size_t)hq_g * d * es;   // bytes per token: all heads / one group
+    for (int g2 = 0; g2 < groups && s == TF_OK; ++g2) {
+        cudaEvent_t ev_q = ctx->ev[3 + 2 * g2], ev_att = ctx->ev[4 + 2 * g2];
+        const size_t off = (size_t)g2 * row_g;
+        e = cudaMemcpy2DAsync(dQ + off, row, static_cast<const char*>(Q_host) + off, row, row_g, tokens, cudaMemcpyHostToDevice, ctx->s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(ev_q, ctx->s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, ev_q, 0);
+        if (e != cudaSuccess) { s = TF_ERR_CUDA; break; }
+        tf_shape gs = *shape;                                  // this group's heads: same strides, fewer heads, shifted bases
+        gs.n_q_heads = hq_g; gs.n_kv_heads = hkv_g;
+        const size_t kv_off = (size_t)g2 * hkv_g * d * es;
+        s = attention_dispatch(ctx, gs, *params, dQ + off, static_cast<char*>(dK) + kv_off, static_cast<char*>(dV) + kv_off, dI, dN,
+                               dO + off, st);
+        if (s != TF_OK) break;
+        e = cudaEventRecord(ev_att, st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_out, ev_att, 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(static_cast<char*>(O_host) + off, row, dO + off, row, row_g, tokens, cudaMemcpyDeviceToHost, ctx->s_out);
+        if (e != cudaSuccess) s = TF_ERR_CUDA;
+    }
     ctx->workspace = saved_ws; ctx->workspace_bytes = saved_bytes;
-    if (s != TF_OK) return s;
-    e = cudaMemcpyAsync(O_host, dO, tokens * shape->n_q_heads * d * es, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess && score_host) e = cudaMemcpyAsync(score_host, dS, tokens * 4, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess && keep_mask_host) e = cudaMemcpyAsync(keep_mask_host, dM, tokens, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess && kept_idx_host) e = cudaMemcpyAsync(kept_idx_host, dI, tokens * 4, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess && n_kept_host) e = cudaMemcpyAsync(n_kept_host, dN, (size_t)shape->batch * 4, cudaMemcpyDeviceToHost, st);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    if (s == TF_OK) {
+        e = cudaStreamWaitEvent(ctx->s_out, ev_sel, 0);
+        if (e == cudaSuccess && score_host) e = cudaMemcpyAsync(score_host, dS, tokens * 4, cudaMemcpyDeviceToHost, ctx->s_out);
+        if (e == cudaSuccess && keep_mask_host) e = cudaMemcpyAsync(keep_mask_host, dM, tokens, cudaMemcpyDeviceToHost, ctx->s_out);
+        if (e == cudaSuccess && kept_idx_host) e = cudaMemcpyAsync(kept_idx_host, dI, tokens * 4, cudaMemcpyDeviceToHost, ctx->s_out);
+        if (e == cudaSuccess && n_kept_host) e = cudaMemcpyAsync(n_kept_host, dN, (size_t)shape->batch * 4, cudaMemcpyDeviceToHost, ctx->s_out);
+        if (e != cudaSuccess) s = TF_ERR_CUDA;
+    }
+    // results are in host memory when the call returns (also drains the internal streams after an error)
+    const cudaError_t e1 = cudaStreamSynchronize(ctx->s_in), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(ctx->s_out);
+    if (s == TF_OK && (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess)) s = TF_ERR_CUDA;
+    return s;
 }
 
 tf_status tf_decode_step(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params, float eta,

@@ -134,6 +134,11 @@ struct tf_ctx {
     size_t stage_bytes;
     void* owned_ws;
     size_t owned_ws_bytes;
+    // ... its copy-in and copy-out streams and the events that chain them with the caller's stream
+    static constexpr int kHostEvents = 3 + 2 * 8;
+    bool host_streams_ready;
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev[kHostEvents];
 };
 
 // ---- per-kernel launchers (defined in the .cu files, called by tf_api.cu) ----------------------

@@ -364,6 +364,28 @@ def test_layer_filter_host_entry_matches_device_entry():
     g.close()
 
 
+@pytest.mark.parametrize("visibility", [tfb.TF_KV_ALL, tfb.TF_KV_RETAINED])
+def test_layer_filter_host_pipelined_head_groups(visibility):
+    """A layer large enough for the host entry point to send Q in groups of query heads (whole KV-head groups)
+    while earlier groups' attention runs and their output rows travel back: same bytes as the device entry point."""
+    q, k, v = _qkv(1, 2048, 32, 8, torch.bfloat16, seed=61)
+    g = Gpu(q, k, v, prune_ratio=0.5, warmup_tokens=4, kv_visibility=visibility)
+    g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
+    torch.cuda.synchronize()
+    qh, kh, vh = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+    oh = torch.full_like(qh, float("nan")).pin_memory()
+    sh = torch.empty(1, 2048).pin_memory(); mh = torch.empty(1, 2048, dtype=torch.uint8).pin_memory()
+    ih = torch.empty(1, 2048, dtype=torch.int32).pin_memory(); nh = torch.empty(1, dtype=torch.int32).pin_memory()
+    hs = tfb.make_shape(qh, kh, vh, oh)
+    for _ in range(2):
+        oh.fill_(float("nan"))
+        g.ctx.tf_layer_filter_host(hs, g.params, qh, kh, vh, oh, sh, mh, ih, nh)
+        assert torch.equal(oh, g.O.cpu()) and torch.equal(sh, g.score.cpu()) and torch.equal(mh, g.keep.cpu())
+        assert torch.equal(ih, g.idx.cpu()) and torch.equal(nh, g.nk.cpu())
+    g.status_ok()
+    g.close()
+
+
 def test_decode_and_prefill_share_the_workspace():
     """The decode step keeps its split-key partial results in the bound workspace, over the region where the
     similarity scan keeps its records; a scan after decode steps must still be right (it clears its region first),
