@@ -6,6 +6,8 @@ same bytes); attention is compared on a seeded sample of (sequence, retained tok
 rows that the oracle computes one by one; the rest is checked through properties that hold at any
 size: pruned rows are exactly zero, retained rows are finite, the kept list is the ascending list of
 the mask's ones padded with -1, and exactly min(E, floor(ratio*S)) tokens are pruned."""
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -20,7 +22,16 @@ DEV = "cuda:0"
 
 @pytest.mark.parametrize("name,layer", [("c2", 0), ("c2", 31), ("c3", 20), ("c4", 16), ("c5", 31)])
 def test_layer_filter_full_size(name, layer):
-    wl = W.WORKLOADS[name]
+    _check_layer(W.WORKLOADS[name], layer)
+
+
+def test_layer_filter_sequence_of_32768_tokens():
+    """Configuration 5's shape at twice its length (two sequences): the selection no longer holds the scores in
+    registers, the scan chains 256 chunks per head, the windowed attention has 128 row blocks per head."""
+    _check_layer(dataclasses.replace(W.WORKLOADS["c5"], name="c5-32k", batch=2, seq=32768), 3)
+
+
+def _check_layer(wl, layer):
     _, q, k, v = next(wl.layer_qkv([layer], DEV))
     B, S, Hq, _ = q.shape
     Hkv = k.shape[2]
