@@ -537,15 +537,21 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             mbar_arrive(bar_p + 8 * i);
         }
         // ---- epilogue: O / l -> bf16 -> the row's token position --------------------------------------
+        // A thread owns a row, and rows of retained tokens lie far apart in O: storing from the registers would
+        // touch 32 different lines per warp instruction.  The rows are therefore staged in the shared memory of the
+        // Q tile (nobody reads it once every MMA has completed; 16-byte chunks XOR-swizzled by the row) and written
+        // out with 16 lanes per 256-byte row.  (maximum, sum) of the split form and the rows' token positions
+        // travel through the first K/V ring slot, equally idle by now.
         if constexpr (kSplit) {
             // merge the two groups' partial results: both accumulators sit in the TMEM lanes of this row,
-            // so each group finishes 64 of the 128 output columns; (maximum, sum) travel through the
-            // shared memory of the Q tile, which nobody reads once every MMA has completed
+            // so each group finishes 64 of the 128 output columns
             mbar_wait(bar_o, 0, abort_flag, p.status, 40);
             __syncwarp();
             tc_fence_after();
-            float2* ml = reinterpret_cast<float2*>(smem + kOffQ);
+            float2* ml = reinterpret_cast<float2*>(smem + kOffRing);
+            int* trow_s = reinterpret_cast<int*>(smem + kOffRing + 4096);
             ml[i * kTileM + r] = make_float2(m_ref, l_run);
+            if (i == 0) trow_s[r] = t_row;                        // -1: no such row
             asm volatile("bar.sync 1, %0;" :: "n"(kSoftmaxThreads) : "memory");
             const float2 other = ml[(i ^ 1) * kTileM + r];
             const bool both = je[1] > jb[1];                       // group 1 had tiles (CTA-uniform)
@@ -556,51 +562,67 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             const float inv = 1.f / (l0 * e0 + l1 * e1);
             const float w0 = e0 * inv, w1 = e1 * inv;
             const uint32_t tm_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-            __nv_bfloat16* orow = Ob + (long long)max(t_row, 0) * p.os.t + i * 64;
+            uint8_t* stage = smem + kOffQ + r * 256;
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t o0[32], o1[32];
                 tmem_ld32(tm_row + 256 + i * 64 + c * 32, o0);
                 if (both) tmem_ld32(tm_row + 384 + i * 64 + c * 32, o1);
                 tmem_wait_ld();
-                if (valid) {
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        float f[8];
+                for (int v = 0; v < 4; ++v) {
+                    float f[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            f[e] = __uint_as_float(o0[8 * v + e]) * w0;
-                            if (both) f[e] = fmaf(__uint_as_float(o1[8 * v + e]), w1, f[e]);
-                        }
-                        uint4 w;
-                        w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
-                        w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
+                    for (int e = 0; e < 8; ++e) {
+                        f[e] = __uint_as_float(o0[8 * v + e]) * w0;
+                        if (both) f[e] = fmaf(__uint_as_float(o1[8 * v + e]), w1, f[e]);
                     }
+                    uint4 w;
+                    w.x = pack_bf16(f[0], f[1]); w.y = pack_bf16(f[2], f[3]);
+                    w.z = pack_bf16(f[4], f[5]); w.w = pack_bf16(f[6], f[7]);
+                    *reinterpret_cast<uint4*>(stage + (((i * 8 + c * 4 + v) ^ (r & 15)) << 4)) = w;
                 }
+            }
+            asm volatile("bar.sync 1, %0;" :: "n"(kSoftmaxThreads) : "memory");
+            const int sub = tid >> 4, l16 = tid & 15;              // 256 threads: 16 rows per pass
+#pragma unroll
+            for (int pass = 0; pass < kTileM / 16; ++pass) {
+                const int R = pass * 16 + sub, t_out = trow_s[R];
+                if (t_out >= 0)
+                    *reinterpret_cast<uint4*>(Ob + (long long)t_out * p.os.t + l16 * 8) =
+                        *reinterpret_cast<const uint4*>(smem + kOffQ + R * 256 + ((l16 ^ (R & 15)) << 4));
             }
         } else if (i < n_q) {
             mbar_wait(bar_o, 0, abort_flag, p.status, 40);
             __syncwarp();
             tc_fence_after();
             const float inv = 1.f / l_run;
-            __nv_bfloat16* orow = Ob + (long long)max(t_row, 0) * p.os.t;
+            int* trow_s = reinterpret_cast<int*>(smem + kOffRing + 4096) + i * kTileM;
+            trow_s[r] = t_row;
+            uint8_t* stage = smem + kOffQ + i * kTileBytes + r * 256;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tm_o + c * 32, o);
                 tmem_wait_ld();
-                if (valid) {
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-                        w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-                        w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-                        w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = w;
-                    }
+                for (int v = 0; v < 4; ++v) {
+                    uint4 w;
+                    w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+                    w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+                    w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+                    w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+                    *reinterpret_cast<uint4*>(stage + (((c * 4 + v) ^ (r & 15)) << 4)) = w;
                 }
+            }
+            asm volatile("bar.sync %0, %1;" :: "r"(2 + i), "n"(kTileM) : "memory");   // this group's 128 threads
+            const int sub = r >> 4, l16 = r & 15;                  // 128 threads: 8 rows per pass
+#pragma unroll
+            for (int pass = 0; pass < kTileM / 8; ++pass) {
+                const int R = pass * 8 + sub, t_out = trow_s[R];
+                if (t_out >= 0)
+                    *reinterpret_cast<uint4*>(Ob + (long long)t_out * p.os.t + l16 * 8) =
+                        *reinterpret_cast<const uint4*>(smem + kOffQ + i * kTileBytes + R * 256 + ((l16 ^ (R & 15)) << 4));
             }
         }
     }
