@@ -347,6 +347,10 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             for (int j = J0; j < J1; ++j) {
                 for (int kv = 0; kv < 2; ++kv, ++q) {
                     const int st = q % kStages;
+                    // the first K and V tiles go out at once; the rest of the ring is filled once the Q rows are in shared
+                    // memory (nothing can consume it earlier, and a ring's worth of arriving tiles keeps the gather's
+                    // shared-memory stores waiting)
+                    if (q == 2) mbar_wait(bar_q, 0, abort_flag, p.status, 11);
                     if (q >= kStages) mbar_wait(bar_empty + 8 * st, ((q / kStages) - 1) & 1, abort_flag, p.status, 10);
                     const uint32_t dst = sbase + kOffRing + st * kTileBytes;
                     const CUtensorMap* map = kv ? &mapV : &mapK;
