@@ -169,6 +169,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    grid_dependency_wait();   // launched so that the set-up above overlaps the tail of the kernel before it on the stream
 
     // Tiles go by block index (K and V of a tile side by side).  CTAs are started in index order, so the
     // records a tile waits for belong to tiles started before it; should a scheduler ever break that order,
@@ -517,6 +518,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         return t < pp.n_tiles ? t : kPNoTile;
     };
 
+    grid_dependency_wait();   // the set-up above overlaps the tail of the kernel before this one on the stream
     if (tid == 0) announce_and_load(draw());
     worker_sync(w);
     uint4 cur = make_uint4(s_next[0], s_next[1], s_next[2], s_next[3]);
@@ -768,13 +770,11 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
         pp.ticket_base = ws->ticket_base;
         pp.n_tiles = n_work;
         ws->ticket_base += n_work + grid * kPWorkers;      // every worker draws once past the end
-        kv_stats_gram_persistent_kernel<<<grid, kPThreads, kPSmem, st>>>(pp, mk, mv);
         ctx->launches += 1;
-        return cudaGetLastError();
+        return launch_dependent(kv_stats_gram_persistent_kernel, dim3(grid), dim3(kPThreads), kPSmem, st, pp, mk, mv);
     }
-    kv_stats_gram1_kernel<<<(unsigned)(2 * tiles), 128, kT1Smem, st>>>(gp, mk, mv);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return launch_dependent(kv_stats_gram1_kernel, dim3((unsigned)(2 * tiles)), dim3(128), kT1Smem, st, gp, mk, mv);
 }
 
 }  // namespace tf
