@@ -42,6 +42,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 dec_from_f<__nv_bfloat16>(f
 template <typename T>
 __global__ void __launch_bounds__(kDecWarps * 32) decode_decide_kernel(const DecideParams p) {
     extern __shared__ float cos_s[];        // [2][Hkv]
+    grid_dependency_wait();                 // launched early; the step before this one on the stream must be complete
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = p.pos[b];
     const long long n0 = p.count[b];
@@ -423,10 +424,10 @@ cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_p
     dp.skips = reinterpret_cast<long long*>(a.state->skips);
     dp.score_out = a.score_out; dp.skip_out = a.skip_out; dp.status = ctx->dev_status;
     const size_t smem = 2 * (size_t)s.n_kv_heads * sizeof(float);
-    if (s.dtype == TF_BF16) decode_decide_kernel<__nv_bfloat16><<<s.batch, kDecWarps * 32, smem, st>>>(dp);
-    else                    decode_decide_kernel<float><<<s.batch, kDecWarps * 32, smem, st>>>(dp);
+    cudaError_t e;
+    if (s.dtype == TF_BF16) e = launch_dependent(decode_decide_kernel<__nv_bfloat16>, dim3((unsigned)s.batch), dim3(kDecWarps * 32), smem, st, dp);
+    else                    e = launch_dependent(decode_decide_kernel<float>, dim3((unsigned)s.batch), dim3(kDecWarps * 32), smem, st, dp);
     ctx->launches += 1;
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
 
     DecAttnParams ap{};
