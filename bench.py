@@ -436,8 +436,8 @@ def main():
         dom = max(names, key=lambda n: per[n])
         # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the ncu
         # captures summarised under profiles/ (50 % pruning, all keys visible); None where none was taken.
-        ncu_traffic = {("c2", "pruned_attention"): 42055424 + 73984, ("c3", "pruned_attention"): 420800256 + 157004800,
-                       ("c3", "kv_stats"): 337403392 + 16380416, ("c2", "kv_stats"): 34768384}
+        ncu_traffic = {("c2", "pruned_attention"): 42053632 + 71680, ("c3", "pruned_attention"): 420844288 + 159603968,
+                       ("c3", "kv_stats"): 337368832 + 15580416, ("c2", "kv_stats"): 34779904 + 256}
         traffic = ncu_traffic.get((wl.name, dom)) if (args.prune == 0.5 and args.kv_visibility == "all") else None
         roof = {"kernel": dom, "bound": kern[dom].get("bound", "latency"), "achieved": kern[dom].get("achieved"),
                 "peak": kern[dom].get("peak"), "unit": kern[dom].get("unit"), "frac": kern[dom].get("frac"),
