@@ -4,15 +4,20 @@
 One step = one pass of the whole hot path (similarity scan, fusion, selection, attention for
 retained tokens) over one layer's Q/K/V of a synthetic, seeded workload.  Prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c1]
-                    [--prune 0.5] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5|c4|c3|c2|c1]
+                    [--prune 0.5] [--impl ours|reference] [--sweep]
+
+The default workload is configuration 5, the largest that fits one GPU (Mistral-7B shape, batch 8 x
+16384 tokens, window 4096).  --sweep prints one line per configuration and pruning ratio and the
+1K-32K sequence sweep of configuration 5.
 
 value   : tokens/s per layer, inputs resident in HBM, timed with CUDA events on the launch stream.
 e2e     : same metric through tf_layer_filter_host (pinned host buffers; copies inside the timing).
 roofline: the dominant kernel against the measured peak of the resource that bounds it.
 cpu_baseline / --impl reference: the fp64 oracle, as it stands, on this machine's host cores.
-N > 1   : one process per GPU (torchrun); sequences are independent, so every rank runs its own
-          replica of the workload with no data-path collective ("weak" scaling).
+N > 1   : one process per GPU (under torchrun, or started from here when no launcher set WORLD_SIZE);
+          sequences are independent, so every rank runs its own replica of the workload with no
+          data-path collective ("weak" scaling).
 """
 from __future__ import annotations
 
@@ -237,7 +242,7 @@ def run_decode(args, wl, tfb, dev, local):
                       "config": workload_config(wl, args), "gpu_launches": int(ctx.launches - launches0),
                       "roofline": {"kernel": "decode_attention", "bound": "hbm", "achieved": cache_bytes / (ms * 1e-3) / 1e9,
                                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": cache_bytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                                   "traffic": {"c5": 134302464 + 602112}.get(wl.name),   # ncu, profiles/decode_step_c5.txt
+                                   "traffic": ncu_traffic(wl.name, "decode_step", 0.0),
                                    "peak_kind": pk_kind, "algorithmic_per_launch": cache_bytes}}))
     ctx.close()
 
@@ -266,44 +271,47 @@ def workload_config(wl, args):
             "l2": "inputs rotate over distinct layers whose total size exceeds the 126 MB L2"}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c2")
-    ap.add_argument("--prune", type=float, default=0.5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kv-visibility", default="all", choices=["all", "retained"],
-                    help="retained: kept queries attend kept keys only (a different, smaller computation)")
-    ap.add_argument("--decode", action="store_true",
-                    help="measure the online decode step (one new token per sequence against a cache of seq tokens) instead")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+def ncu_traffic(workload: str, kernel: str, prune: float):
+    """DRAM bytes per launch (read + write) of a kernel from the ncu summaries: profiles/dram_traffic.txt holds one
+    line per capture, `workload kernel prune read_bytes write_bytes`; None where no capture was taken."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        f = line.split()
+        if len(f) >= 5 and not line.startswith("#") and f[0] == workload and f[1] == kernel and abs(float(f[2]) - prune) < 1e-9:
+            return int(f[3]) + int(f[4])
+    return None
 
-    from paper_2512_07090_b200 import workloads as W
-    wl = W.WORKLOADS[args.workload]
-    if args.impl == "reference":
-        run_reference(args, wl)
-        return
 
-    from paper_2512_07090_b200 import binding as tfb
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = f"cuda:{local}"
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-    wl.seed = rank_seed(wl.seed, rank)
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # the figures the targets are stated against
 
-    tfb.lib()   # fails loudly if the CUDA library is not built
-    if args.decode:
-        run_decode(args, wl, tfb, dev, local)
-        return
+
+def timed_repeats(fn, steps, sync_all, dist, dev, min_total_ms=300.0, max_repeats=200):
+    """Times `steps` calls of fn(i) between two CUDA events, several times over (each repeat bracketed by a
+    synchronise, and a barrier when there are ranks), until the timed work adds up to min_total_ms, so that the
+    clock sampler sees the GPU under this load; returns (median ms of one repeat, all repeats, slowest rank each)."""
+    times = []
+    repeats = 3
+    i0 = 0
+    while len(times) < repeats:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sync_all()
+        e0.record()
+        for i in range(steps):
+            fn(i0 + i)
+        e1.record()
+        sync_all()
+        i0 += steps
+        times.append(max_over_ranks(e0.elapsed_time(e1), dist, dev))
+        if len(times) == 1:   # the same count on every rank: it comes from the slowest rank's first repeat
+            repeats = int(min(max_repeats, max(3, -(-min_total_ms // max(times[0], 1e-3)))))
+    return statistics.median(times), times
+
+
+def measure(wl, args, tfb, dev, local, dist, world, rank, headline=True):
+    """One workload at one pruning ratio: the whole layer step, each stage alone, and (headline only) the host-buffer
+    entry point and the oracle on host cores.  Returns the JSON object of the line (rank 0) or None."""
     ring = make_ring(wl, dev, min_bytes=300 << 20)
     B, S, Hq, d = ring[0][0].shape
     Hkv = ring[0][1].shape[2]
@@ -336,20 +344,15 @@ def main():
     code, det = ctx.tf_get_status()
     if code != tfb.TF_OK:
         raise RuntimeError(f"device status {code}: {det}")
+    scan_kernel, attn_kernel = ctx.tf_last_kernels()
 
-    # ---- timed region: K whole steps --------------------------------------------------------------
+    # ---- timed region: K whole steps, repeated; the median repeat is the figure -----------------------
     sampler = ClockSampler(local)
     sampler.start()
     l0 = ctx.launches
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync_all()
-    e0.record()
-    for i in range(args.steps):
-        step(args.warmup + i)
-    e1.record()
-    sync_all()
-    ms = e0.elapsed_time(e1)
-    launches = ctx.launches - l0
+    ms, reps = timed_repeats(step, args.steps, sync_all, dist, dev)
+    launches = (ctx.launches - l0) // len(reps)
+    busy_ms = sum(reps)
 
     # ---- per-kernel durations: each stage entry point alone, K launches back to back ---------------
     # (events around the whole loop, so launch latency is not charged to the kernel; every ring entry
@@ -380,80 +383,197 @@ def main():
     for n in names:
         for i in range(3):
             stage(n, i)
-        torch.cuda.synchronize()
-        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s0.record()
-        for i in range(args.steps):
-            stage(n, args.warmup + i)
-        s1.record()
-        torch.cuda.synchronize()
-        per[n] = s0.elapsed_time(s1) / args.steps
+        t, _ = timed_repeats(lambda i, n=n: stage(n, i), args.steps, sync_all, None, dev, min_total_ms=100.0)
+        per[n] = t / args.steps
     clocks = sampler.stop()
 
-    ms = max_over_ranks(ms, dist, dev)
     tokens_per_step = B * S * world
     value = tokens_per_step * args.steps / (ms * 1e-3)
 
     # ---- end to end through the host entry point ----------------------------------------------------
-    qh, kh, vh = (t.cpu().pin_memory() for t in ring[0])
-    oh = torch.empty_like(qh).pin_memory()
-    nh = torch.empty(B, dtype=torch.int32).pin_memory()
-    hshape = tfb.make_shape(qh, kh, vh, oh, window=wl.window)
-    e2e_steps = max(3, min(args.steps, 10))
-    for _ in range(2):
-        ctx.tf_layer_filter_host(hshape, params, qh, kh, vh, oh, None, None, None, nh)
-    sync_all()
-    t0 = time.perf_counter()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for _ in range(e2e_steps):
-        ctx.tf_layer_filter_host(hshape, params, qh, kh, vh, oh, None, None, None, nh)
-    f1.record()
-    sync_all()
-    e2e_ms = f0.elapsed_time(f1)
-    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
-    e2e = {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
-           "h2d_bytes_per_step": int((qh.numel() + kh.numel() + vh.numel()) * es),
-           "d2h_bytes_per_step": int(oh.numel() * es + nh.numel() * 4), "steps": e2e_steps}
+    e2e = None
+    if headline:
+        qh, kh, vh = (t.cpu().pin_memory() for t in ring[0])
+        oh = torch.empty_like(qh).pin_memory()
+        nh = torch.empty(B, dtype=torch.int32).pin_memory()
+        hshape = tfb.make_shape(qh, kh, vh, oh, window=wl.window)
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            ctx.tf_layer_filter_host(hshape, params, qh, kh, vh, oh, None, None, None, nh)
+        sync_all()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(e2e_steps):
+            ctx.tf_layer_filter_host(hshape, params, qh, kh, vh, oh, None, None, None, nh)
+        f1.record()
+        sync_all()
+        e2e_ms = max_over_ranks(f0.elapsed_time(f1), dist, dev)
+        e2e = {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int((qh.numel() + kh.numel() + vh.numel()) * es),
+               "d2h_bytes_per_step": int(oh.numel() * es + nh.numel() * 4), "steps": e2e_steps}
+        del qh, kh, vh, oh
 
+    out = None
     if rank == 0:
         pk, pk_kind = peaks()
         kv_bytes = 2.0 * B * S * Hkv * d * es + 8.0 * B * S * Hkv
-        kern = {}
-        for n in names:
-            kern[n] = {"us": per[n] * 1e3}
-        kern["kv_stats"].update(bound="hbm", achieved=kv_bytes / (per["kv_stats"] * 1e-3) / 1e9, unit="GB/s",
-                                peak=pk["hbm_gbs"])
-        kern["kv_stats"]["frac"] = kern["kv_stats"]["achieved"] / pk["hbm_gbs"]
-        long_run = ms > 2000.0
+        sel_bytes = (4.0 * Hkv * 2 + 4.0) * B * S + 9.0 * B * S          # fusion: sims in, score out; selection: score in, mask + index out
+        kern = {n: {"us": per[n] * 1e3} for n in names}
+        kv = kern["kv_stats"]
+        kv.update(bound="hbm", achieved=kv_bytes / (per["kv_stats"] * 1e-3) / 1e9, unit="GB/s", peak=pk["hbm_gbs"])
+        kv["frac"] = kv["achieved"] / pk["hbm_gbs"]
+        kv["frac_of_nominal"] = kv["achieved"] / NOMINAL["hbm_gbs"]
+        # scoring + selection together (steps a1-a4): their bytes over the sum of their times
+        t_filter = per["kv_stats"] + per["score_fuse"] + per["select"]
+        ach_f = (kv_bytes + sel_bytes) / (t_filter * 1e-3) / 1e9
+        kern["scoring_and_selection"] = {"us": t_filter * 1e3, "bound": "hbm", "achieved": ach_f, "unit": "GB/s",
+                                         "peak": pk["hbm_gbs"], "frac": ach_f / pk["hbm_gbs"],
+                                         "frac_of_nominal": ach_f / NOMINAL["hbm_gbs"]}
+        long_run = busy_ms > 2000.0
         tpeak = pk["bf16_tflops_sustained"] if long_run else pk["bf16_tflops"]
         ach = flops / (per["pruned_attention"] * 1e-3) / 1e12
+        pa = kern["pruned_attention"]
         if wl.dtype == torch.bfloat16:
-            kern["pruned_attention"].update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tpeak, frac=ach / tpeak)
-        else:
-            kern["pruned_attention"].update(bound="alu", achieved=ach, unit="TFLOP/s", peak=148 * 128 * 2 * 1.965e-3,
-                                            frac=ach / (148 * 128 * 2 * 1.965e-3))
+            pa.update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tpeak, frac=ach / tpeak,
+                      frac_of_burst=ach / pk["bf16_tflops"], frac_of_sustained=ach / pk["bf16_tflops_sustained"],
+                      frac_of_nominal=ach / NOMINAL["bf16_tflops"])
+        else:   # fp32 on the CUDA cores: 148 SMs x 128 lanes x 2 flop x max clock
+            alu = 148 * 128 * 2 * 1.965e-3
+            pa.update(bound="alu", achieved=ach, unit="TFLOP/s", peak=alu, frac=ach / alu)
         dom = max(names, key=lambda n: per[n])
-        # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the ncu
-        # captures summarised under profiles/ (50 % pruning, all keys visible); None where none was taken.
-        ncu_traffic = {("c2", "pruned_attention"): 42053632 + 71680, ("c3", "pruned_attention"): 420844288 + 159603968,
-                       ("c3", "kv_stats"): 337368832 + 15580416, ("c2", "kv_stats"): 34779904 + 256}
-        traffic = ncu_traffic.get((wl.name, dom)) if (args.prune == 0.5 and args.kv_visibility == "all") else None
+        traffic = ncu_traffic(wl.name, dom, args.prune) if args.kv_visibility == "all" else None
         roof = {"kernel": dom, "bound": kern[dom].get("bound", "latency"), "achieved": kern[dom].get("achieved"),
                 "peak": kern[dom].get("peak"), "unit": kern[dom].get("unit"), "frac": kern[dom].get("frac"),
                 "traffic": traffic, "peak_kind": f"{pk_kind} ({'sustained' if long_run else 'burst'} bf16)" if dom == "pruned_attention" else pk_kind,
                 "algorithmic_per_launch": flops if dom == "pruned_attention" else kv_bytes}
+        cfg = workload_config(wl, args)
+        cfg["timing"] = (f"median of {len(reps)} repeats of {args.steps} steps ({busy_ms:.0f} ms timed in all); "
+                         f"per-kernel: each stage alone, same scheme")
+        cfg["kernels_chosen"] = {"scan": scan_kernel, "attention": attn_kernel}
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16" if wl.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-               "config": workload_config(wl, args), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-               "roofline": roof, "kernels": kern}
-        if not args.no_cpu_baseline and world == 1 and args.kv_visibility == "all":   # the baseline arm times the default reading
+               "config": cfg, "clocks": clocks, "gpu_launches": int(launches), "roofline": roof, "kernels": kern}
+        if e2e is not None:
+            out["e2e"] = e2e
+        if headline and not args.no_cpu_baseline and world == 1 and args.kv_visibility == "all":   # the baseline arm times the default reading
             q, k, v = ring[0]
             out["cpu_baseline"] = oracle_sample(wl, (q.float().cpu().numpy(), k.float().cpu().numpy(),
                                                      v.float().cpu().numpy()), args.prune)
-        print(json.dumps(out))
+            out["cpu_baseline"]["c1_whole_layer_s"] = oracle_c1_times()
     ctx.close()
+    del ring, state
+    torch.cuda.empty_cache()
+    return out
+
+
+def oracle_c1_times():
+    """Configuration 1 (B1 S128, 32 heads, fp32, 50 % pruning) through the whole oracle, on one thread and on all."""
+    import oracle
+    from paper_2512_07090_b200 import workloads as W
+    wl = W.WORKLOADS["c1"]
+    _, q, k, v = next(wl.layer_qkv([0], "cpu"))
+    q, k, v = q.numpy(), k.numpy(), v.numpy()
+    n_all = oracle.num_threads()
+    res = {}
+    for label, n in (("threads_1", 1), (f"threads_{n_all}", n_all)):
+        oracle.set_num_threads(n)
+        oracle.layer_filter(q, k, v, prune_ratio=0.5, warmup_tokens=4)
+        t0 = time.perf_counter()
+        for _ in range(5):
+            oracle.layer_filter(q, k, v, prune_ratio=0.5, warmup_tokens=4)
+        res[label] = (time.perf_counter() - t0) / 5
+    oracle.set_num_threads(n_all)
+    return res
+
+
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU, torchrun's
+    environment, rendezvous on 127.0.0.1) with the same arguments and return their exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd).returncode
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c5",
+                    help="c1..c5; the default is the largest single-GPU configuration (Mistral-7B shape, batch 8 x 16384 tokens, window 4096)")
+    ap.add_argument("--prune", type=float, default=0.5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv-visibility", default="all", choices=["all", "retained"],
+                    help="retained: kept queries attend kept keys only (a different, smaller computation)")
+    ap.add_argument("--decode", action="store_true",
+                    help="measure the online decode step (one new token per sequence against a cache of seq tokens) instead")
+    ap.add_argument("--sweep", action="store_true",
+                    help="one line per configuration and pruning ratio (c1-c5), then configuration 5 at 1K-32K tokens; "
+                         "device-resident figures only")
+    ap.add_argument("--backend", default="nccl", help="process-group backend of an N > 1 run (gloo: CPU-only test of the launch path)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
+
+    from paper_2512_07090_b200 import workloads as W
+    wl = W.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.backend == "gloo":      # launch-path check without GPUs: ranks, seeds, barrier, max over ranks, one line
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        seed = rank_seed(wl.seed, rank)
+        slow = max_over_ranks(1.0 + rank, dist, "cpu")
+        dist.barrier()
+        if rank == 0:
+            print(json.dumps({"launch_check": True, "n_gpus": world, "slowest_ms": slow, "seed_rank0": seed,
+                              "config": workload_config(wl, args)}))
+        dist.destroy_process_group()
+        return
+
+    from paper_2512_07090_b200 import binding as tfb
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    import dataclasses
+    base_seed = {n: w.seed for n, w in W.WORKLOADS.items()}
+    wl = dataclasses.replace(wl, seed=rank_seed(wl.seed, rank))
+
+    tfb.lib()   # fails loudly if the CUDA library is not built
+    if args.decode:
+        run_decode(args, wl, tfb, dev, local)
+        return
+    if args.sweep:
+        seeded = {n: dataclasses.replace(w, seed=rank_seed(base_seed[n], rank)) for n, w in W.WORKLOADS.items()}
+        cases = [(seeded[n], r) for n in ("c1", "c2", "c3", "c4", "c5") for r in seeded[n].prune_ratios]
+        cases += [(dataclasses.replace(seeded["c5"], name=f"c5-s{s // 1024}k", seq=s), 0.5)
+                  for s in (1024, 2048, 4096, 8192, 16384, 32768)]
+        for w, r in cases:
+            a = argparse.Namespace(**vars(args)); a.prune = r
+            out = measure(w, a, tfb, dev, local, dist, world, rank, headline=False)
+            if out is not None:
+                out["sweep"] = True
+                print(json.dumps(out), flush=True)
+    else:
+        out = measure(wl, args, tfb, dev, local, dist, world, rank, headline=True)
+        if out is not None:
+            print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
 

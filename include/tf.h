@@ -55,7 +55,7 @@ enum { TF_ANCHOR_PAST_MEAN = 0, /* tokens strictly before t (default)           
 /* fuse_mode: the weight alpha of Eq. 2-3 */
 enum { TF_FUSE_INVVAR = 0,      /* alpha = var_v/(var_k+var_v): lower variance weighs more */
        TF_FUSE_EQ2_LITERAL = 1, /* alpha = var_k/(var_k+var_v): Eq. 2 exactly as printed   */
-       TF_FUSE_KEY_ONLY = 2, TF_FUSE_VALUE_ONLY = 3, /* criterion ablation (Section 4.4)   */
+       TF_FUSE_KEY_ONLY = 2, TF_FUSE_VALUE_ONLY = 3, /* criterion ablation (Section 4.3)   */
        TF_FUSE_MEAN = 4 };      /* alpha = 1/2 (Figure 1 caption)                          */
 enum { TF_SELECT_RATIO = 0,     /* prune exactly P = min(E, floor(ratio*S)) top-scoring eligible tokens */
        TF_SELECT_THRESHOLD = 1 }; /* prune eligible tokens with score > threshold (strict) */
@@ -131,9 +131,10 @@ tf_status tf_kv_stats(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params
  *     device, and device-side conditions (a wait that gave up) are recorded in it.  With NULL
  *     they are not recorded anywhere.
  *   - Limit: shapes whose records need more than TF_STATIC_SCRATCH_BYTES return
- *     TF_ERR_WORKSPACE and launch nothing.  The records take 2 KiB per (64 tokens (bf16) or
- *     32 tokens (fp32), sequence, KV head) plus one eighth of that; 8 MiB covers, for example,
- *     batch 1 x 2048 tokens x 32 KV heads in bf16 three times over.
+ *     TF_ERR_WORKSPACE and launch nothing.  The need is that of the largest record layout any
+ *     scan kernel may use for the shape: 2 KiB per (64 tokens (bf16) or 32 tokens (fp32),
+ *     sequence, KV head) plus one eighth of that; 8 MiB covers, for example, batch 1 x 2048
+ *     tokens x 32 KV heads in bf16 three times over.
  *   - The first call on each device looks up the array's device address and zeroes the part
  *     it uses; make that first call outside any stream capture.
  *   - Every GPU on which the library is loaded holds the array until the process exits.
@@ -235,22 +236,45 @@ tf_status tf_tail_policy(double p_global, double tail_fraction, int32_t n_layers
 
 /* Device-side conditions since the last tf_clear_status: returns TF_OK, TF_ERR_TIMEOUT or
  * TF_ERR_NAN_SCORE.  sync != 0 synchronises the device first.  detail (may be NULL) receives
- * four words: {code, where, count of NaN scores, kernels launched by this context}. */
+ * four words: {code, where, count of NaN scores, kernels launched by this context}.  After a
+ * TF_ERR_TIMEOUT the outputs of the call that saw it are undefined; the context stays usable
+ * (the next similarity scan clears its scratch records first). */
 tf_status tf_get_status(tf_ctx *ctx, int sync, int64_t detail[4]);
 tf_status tf_clear_status(tf_ctx *ctx);
 
+/* Which kernel ran.  kernels[0] = the kernel of the latest similarity scan (steps a1+a2) launched
+ * through this context, kernels[1] = the kernel of the latest attention (step a5); TF_KERNEL_NONE
+ * before the first. */
+enum { TF_KERNEL_NONE = 0,
+       TF_KERNEL_SCAN_PLAIN = 1,            /* CUDA-core chained scan (fp32 inputs, EMA anchors)      */
+       TF_KERNEL_SCAN_GRAM_TILE = 2,        /* tcgen05 Gram-matrix scan, one tile per CTA             */
+       TF_KERNEL_SCAN_GRAM_PERSISTENT = 3,  /* tcgen05 Gram-matrix scan, persistent                   */
+       TF_KERNEL_ATTN_SIMT = 10,            /* CUDA-core attention (fp32)                             */
+       TF_KERNEL_ATTN_TC_SHARED = 11,       /* tcgen05 attention, two Q tiles share every K/V tile    */
+       TF_KERNEL_ATTN_TC_SPLIT = 12 };      /* tcgen05 attention, one Q tile, K/V tiles split         */
+tf_status tf_last_kernels(tf_ctx *ctx, int32_t kernels[2]);
+
 /* Which attention kernel a bf16 call uses: 1 = tcgen05 tensor-core kernel (default; it picks between
- * its two work distributions by problem size), 0 = the plain CUDA-core kernel that fp32 always uses,
- * 2 = tensor-core kernel, two Q tiles per CTA sharing every K/V tile, 3 = tensor-core kernel, one Q
- * tile per CTA with its K/V tiles split between the CTA's two softmax groups.  For A/B checks. */
+ * its two work distributions by problem size; if no tensor map can describe the caller's K/V layout it
+ * uses the CUDA-core kernel), 0 = the plain CUDA-core kernel that fp32 always uses, 2 = tensor-core
+ * kernel, two Q tiles per CTA sharing every K/V tile, 3 = tensor-core kernel, one Q tile per CTA with its
+ * K/V tiles split between the CTA's two softmax groups.  With 2 or 3 the named kernel is a requirement:
+ * a call it cannot take fails with TF_ERR_UNSUPPORTED instead of running another kernel.  For A/B checks. */
 tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
 
 /* Which kernel tf_kv_stats uses: 0 = choose (default: by dtype, anchor mode and problem size), 1 = the
  * plain CUDA-core kernel (any dtype and anchor mode), 2 = the kernel that forms 128-token Gram matrices
  * on the tensor cores, one tile per CTA, 3 = the same arithmetic as a persistent kernel (one CTA per SM,
  * six tiles in flight).  2 and 3 take bf16 with running-sum anchors; other calls then fail with
- * TF_ERR_CUDA.  For A/B checks. */
+ * TF_ERR_UNSUPPORTED.  For A/B checks. */
 tf_status tf_set_scan_path(tf_ctx *ctx, int path);
+
+/* Limits of the bounded waits inside the kernels (every wait on another CTA's record or on an mbarrier
+ * gives up after its limit, records TF_ERR_TIMEOUT and lets the kernel finish).  max_polls: how often one
+ * look-back record is re-read before giving up (0: a record that is not there at the first look counts as
+ * missing); wait_cycles: SM clock cycles one mbarrier wait may take.  A negative value restores the
+ * default (about a second each).  For tests of the error path and for deployments that want a tighter bound. */
+tf_status tf_set_wait_limits(tf_ctx *ctx, int64_t max_polls, int64_t wait_cycles);
 
 const char *tf_status_string(tf_status s);
 

@@ -228,10 +228,9 @@ def decode_step(state, q, K_cache, V_cache, pos, target_ratio=0.5, eta=0.05, war
         s = float(score_fuse(ck[None, None, :], cv[None, None, :], fuse_mode, var_eps)[0, 0])
         steps, skips = int(state["steps"][b]), int(state["skips"][b])
         rho = skips / steps if steps > 0 else 0.0
-        e32, t32 = float(np.float32(eta)), float(np.float32(target_ratio))   # the kernel holds these two in fp32
-        delta = e32 * ((t32 - rho) if alg1_sign else (rho - t32))
-        state["tau"][b] = np.float32(np.float32(state["tau"][b]) + np.float32(delta))   # the threshold is kept in fp32
-        decide = bool(np.float32(s) > state["tau"][b]) if s == s else False
+        delta = eta * ((target_ratio - rho) if alg1_sign else (rho - target_ratio))
+        state["tau"][b] = state["tau"][b] + delta
+        decide = bool(s > state["tau"][b]) if s == s else False
         do_skip = decide and pos[b] >= warmup_tokens
         state["steps"][b] = steps + 1
         state["skips"][b] = skips + (1 if decide else 0)

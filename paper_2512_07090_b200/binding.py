@@ -24,11 +24,14 @@ TF_FUSE_INVVAR, TF_FUSE_EQ2_LITERAL, TF_FUSE_KEY_ONLY, TF_FUSE_VALUE_ONLY, TF_FU
 TF_SELECT_RATIO, TF_SELECT_THRESHOLD = 0, 1
 TF_KV_ALL, TF_KV_RETAINED = 0, 1
 TF_STATIC_SCRATCH_BYTES = 8 << 20
+(TF_KERNEL_NONE, TF_KERNEL_SCAN_PLAIN, TF_KERNEL_SCAN_GRAM_TILE, TF_KERNEL_SCAN_GRAM_PERSISTENT) = range(4)
+TF_KERNEL_ATTN_SIMT, TF_KERNEL_ATTN_TC_SHARED, TF_KERNEL_ATTN_TC_SPLIT = 10, 11, 12
 
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
-           "tf_status_string", "tf_tail_policy", "tf_decode_step", "tf_set_scan_path")
+           "tf_status_string", "tf_tail_policy", "tf_decode_step", "tf_set_scan_path", "tf_last_kernels",
+           "tf_set_wait_limits")
 
 
 class tf_shape(C.Structure):
@@ -241,6 +244,17 @@ class Context:
     def tf_set_scan_path(self, path: int):
         """0: choose; 1: plain CUDA-core similarity scan; 2: Gram-matrix scan on the tensor cores (bf16 sums), one tile per CTA; 3: the same, persistent."""
         _check(lib().tf_set_scan_path(self._h, C.c_int(int(path))), "tf_set_scan_path")
+
+    def tf_last_kernels(self):
+        """(kernel of the latest similarity scan, kernel of the latest attention) as TF_KERNEL_* ids."""
+        out = (C.c_int32 * 2)()
+        _check(lib().tf_last_kernels(self._h, out), "tf_last_kernels")
+        return int(out[0]), int(out[1])
+
+    def tf_set_wait_limits(self, max_polls: int = -1, wait_cycles: int = -1):
+        """Limits of the kernels' bounded waits (negative: the default, about a second)."""
+        _check(lib().tf_set_wait_limits(self._h, C.c_int64(int(max_polls)), C.c_int64(int(wait_cycles))),
+               "tf_set_wait_limits")
 
     @property
     def launches(self) -> int:

@@ -21,7 +21,7 @@ WsLayout ws_layout(const tf_shape& s, const tf_filter_params* p) {
     WsLayout w{};
     const size_t tokens = (size_t)s.batch * (size_t)s.seq;
     size_t off = 0;
-    w.scan = off;      off += scan_plan(s).bytes;
+    w.scan = off;      off += scan_scratch_bytes(s);   // whichever scan kernel gets picked
     w.sim_k = off;     off += align256(tokens * s.n_kv_heads * sizeof(float));
     w.sim_v = off;     off += align256(tokens * s.n_kv_heads * sizeof(float));
     w.score = off;     off += align256(tokens * sizeof(float));
@@ -86,21 +86,40 @@ struct DeviceGuard {
     int target = -1;
 };
 
+// NotSupported is how a launcher says "this call is outside what my kernel takes"
+tf_status to_status(cudaError_t e) {
+    return e == cudaSuccess ? TF_OK : (e == cudaErrorNotSupported ? TF_ERR_UNSUPPORTED : TF_ERR_CUDA);
+}
+
+// after a bounded wait gave up, or a launch failed, the records of every scan scratch this context knows are suspect
+void invalidate_scan_scratch(tf_ctx* ctx) {
+    ctx->scan_user.needs_clear = true;
+    ctx->scan_owned.needs_clear = true;
+    tf::static_scratch_invalidate(ctx->device);
+}
+
+// kv_compact: TF_KV_RETAINED on the tensor-core path only -- kv_compact_bytes(shape of the WHOLE call) bytes in the
+// bound workspace (a call on a group of heads reuses the front of it)
 tf_status attention_dispatch(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const void* Q,
                              const void* K, const void* V, const int32_t* kept_idx,
-                             const int32_t* n_kept, void* O, cudaStream_t st) {
-    cudaError_t e = cudaErrorNotSupported;
+                             const int32_t* n_kept, void* O, void* kv_compact, cudaStream_t st) {
     if (s.dtype == TF_BF16 && ctx->use_tensor_cores) {
-        void* kv_compact = nullptr;
-        if (p.kv_visibility == TF_KV_RETAINED) {   // needs the workspace section for the retained K / V
-            const WsLayout w = ws_layout(s, &p);
-            if (!ctx->workspace || ctx->workspace_bytes < w.total) return TF_ERR_WORKSPACE;
-            kv_compact = static_cast<char*>(ctx->workspace) + w.kv_compact;
-        }
-        e = launch_attention_tc(ctx, s, p, Q, K, V, kept_idx, n_kept, O, kv_compact, st);
+        const cudaError_t e = launch_attention_tc(ctx, s, p, Q, K, V, kept_idx, n_kept, O, kv_compact, st);
+        // The default path falls back to the CUDA-core kernel only when no tensor map can describe the caller's
+        // layout; an explicitly requested form is a requirement, and any other failure is an error.
+        if (e != cudaErrorNotSupported || ctx->attention_form != 0) return to_status(e);
     }
-    if (e == cudaErrorNotSupported) e = launch_attention_simt(ctx, s, p, Q, K, V, kept_idx, n_kept, O, st);
-    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    return to_status(launch_attention_simt(ctx, s, p, Q, K, V, kept_idx, n_kept, O, st));
+}
+
+// the workspace section for the retained tokens' K / V, or nullptr when this call does not need one
+tf_status kv_compact_section(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, void** out) {
+    *out = nullptr;
+    if (p.kv_visibility != TF_KV_RETAINED || s.dtype != TF_BF16 || !ctx->use_tensor_cores) return TF_OK;
+    const WsLayout w = ws_layout(s, &p);
+    if (!ctx->workspace || ctx->workspace_bytes < w.total) return TF_ERR_WORKSPACE;
+    *out = static_cast<char*>(ctx->workspace) + w.kv_compact;
+    return TF_OK;
 }
 
 }  // namespace
@@ -131,6 +150,8 @@ tf_status tf_create(tf_ctx** out, int device) {
     if (!c) return TF_ERR_CUDA;
     c->device = device;
     c->use_tensor_cores = 1;
+    c->max_polls = -1;
+    c->wait_cycles = -1;
     if (cudaMalloc(reinterpret_cast<void**>(&c->dev_status), sizeof(DevStatus)) != cudaSuccess ||
         cudaMemset(c->dev_status, 0, sizeof(DevStatus)) != cudaSuccess) {
         delete c;
@@ -170,6 +191,7 @@ tf_status tf_set_workspace(tf_ctx* ctx, void* device_ptr, size_t bytes) {
     ctx->workspace_bytes = device_ptr ? bytes : 0;
     ctx->scan_user = tf::ScanScratch();
     ctx->scan_user.ptr = device_ptr;
+    ctx->scan_user.capacity = ctx->workspace_bytes;
     return TF_OK;
 }
 
@@ -182,12 +204,11 @@ tf_status tf_kv_stats(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params
     if (s == TF_OK) s = check_kv(shape, K, V);
     if (s != TF_OK) return s;
     if (!sim_k || !sim_v) return TF_ERR_INVALID_ARG;
-    if (!ctx->workspace || ctx->workspace_bytes < scan_plan(*shape).bytes) return TF_ERR_WORKSPACE;
+    if (!ctx->workspace || ctx->workspace_bytes < scan_scratch_bytes(*shape)) return TF_ERR_WORKSPACE;
     DeviceGuard g(ctx->device);
     if (!g.ok) return TF_ERR_CUDA;
-    cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, carry, &ctx->scan_user,
-                                    static_cast<cudaStream_t>(stream));
-    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    return to_status(launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, carry, &ctx->scan_user,
+                                     static_cast<cudaStream_t>(stream)));
 }
 
 tf_status tf_score_fuse(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params,
@@ -200,7 +221,7 @@ tf_status tf_score_fuse(tf_ctx* ctx, const tf_shape* shape, const tf_filter_para
     DeviceGuard g(ctx->device);
     if (!g.ok) return TF_ERR_CUDA;
     cudaError_t e = launch_score_fuse(ctx, *shape, *params, sim_k, sim_v, score, static_cast<cudaStream_t>(stream));
-    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    return to_status(e);
 }
 
 tf_status tf_select(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params,
@@ -231,7 +252,10 @@ tf_status tf_pruned_attention(tf_ctx* ctx, const tf_shape* shape, const tf_filte
     if (!stride_ok(shape->q_stride, shape->dtype) || !stride_ok(shape->o_stride, shape->dtype)) return TF_ERR_UNSUPPORTED;
     DeviceGuard g(ctx->device);
     if (!g.ok) return TF_ERR_CUDA;
-    return attention_dispatch(ctx, *shape, *params, Q, K, V, kept_idx, n_kept, O, static_cast<cudaStream_t>(stream));
+    void* kv_compact = nullptr;
+    s = kv_compact_section(ctx, *shape, *params, &kv_compact);
+    if (s != TF_OK) return s;
+    return attention_dispatch(ctx, *shape, *params, Q, K, V, kept_idx, n_kept, O, kv_compact, static_cast<cudaStream_t>(stream));
 }
 
 tf_status tf_layer_filter(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params,
@@ -264,8 +288,11 @@ tf_status tf_layer_filter(tf_ctx* ctx, const tf_shape* shape, const tf_filter_pa
     cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, nullptr, scan, st);
     if (e == cudaSuccess) e = launch_score_fuse(ctx, *shape, *params, sim_k, sim_v, score, st);
     if (e == cudaSuccess) e = launch_select(ctx, *shape, *params, score, keep_mask, kept_idx, n_kept, theta, st);
-    if (e != cudaSuccess) return TF_ERR_CUDA;
-    return attention_dispatch(ctx, *shape, *params, Q, K, V, kept_idx, n_kept, O, st);
+    if (e != cudaSuccess) return to_status(e);
+    void* kv_compact = nullptr;
+    s = kv_compact_section(ctx, *shape, *params, &kv_compact);
+    if (s != TF_OK) return s;
+    return attention_dispatch(ctx, *shape, *params, Q, K, V, kept_idx, n_kept, O, kv_compact, st);
 }
 
 tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params,
@@ -306,6 +333,7 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         ctx->owned_ws_bytes = w.total;
         ctx->scan_owned = tf::ScanScratch();
         ctx->scan_owned.ptr = ctx->owned_ws;
+        ctx->scan_owned.capacity = ctx->owned_ws_bytes;
     }
     char* base = static_cast<char*>(ctx->stage);
     char* dQ = base; char* dO = base + qb; void* dK = base + 2 * qb; void* dV = base + 2 * qb + kb;
@@ -356,7 +384,9 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         if (e == cudaSuccess) e = launch_select(ctx, ds, *params, dS, dM, dI, dN, theta, st);
         if (e == cudaSuccess) e = cudaEventRecord(ev_sel, st);
     }
-    s = e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    s = to_status(e);
+    void* kv_compact = nullptr;                                // the whole call's section: every head group reuses its front
+    if (s == TF_OK) s = kv_compact_section(ctx, *shape, *params, &kv_compact);
     const size_t row = (size_t)shape->n_q_heads * d * es, row_g = (size_t)hq_g * d * es;   // bytes per token: all heads / one group
     for (int g2 = 0; g2 < groups && s == TF_OK; ++g2) {
         cudaEvent_t ev_q = ctx->ev[3 + 2 * g2], ev_att = ctx->ev[4 + 2 * g2];
@@ -369,7 +399,7 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         gs.n_q_heads = hq_g; gs.n_kv_heads = hkv_g;
         const size_t kv_off = (size_t)g2 * hkv_g * d * es;
         s = attention_dispatch(ctx, gs, *params, dQ + off, static_cast<char*>(dK) + kv_off, static_cast<char*>(dV) + kv_off, dI, dN,
-                               dO + off, st);
+                               dO + off, kv_compact, st);
         if (s != TF_OK) break;
         e = cudaEventRecord(ev_att, st);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_out, ev_att, 0);
@@ -439,7 +469,10 @@ tf_status tf_get_status(tf_ctx* ctx, int sync, int64_t detail[4]) {
         detail[0] = (int64_t)h.code; detail[1] = (int64_t)h.where;
         detail[2] = (int64_t)h.nan_count; detail[3] = (int64_t)ctx->launches;
     }
-    if (h.code == TF_ERR_TIMEOUT) return TF_ERR_TIMEOUT;
+    if (h.code == TF_ERR_TIMEOUT) {
+        invalidate_scan_scratch(ctx);   // records written under a wait that gave up are not to be trusted
+        return TF_ERR_TIMEOUT;
+    }
     if (h.code == TF_ERR_NAN_SCORE) return TF_ERR_NAN_SCORE;
     return TF_OK;
 }
@@ -448,7 +481,22 @@ tf_status tf_clear_status(tf_ctx* ctx) {
     if (!ctx) return TF_ERR_INVALID_ARG;
     DeviceGuard g(ctx->device);
     if (!g.ok) return TF_ERR_CUDA;
+    invalidate_scan_scratch(ctx);
     return cudaMemset(ctx->dev_status, 0, sizeof(DevStatus)) == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+}
+
+tf_status tf_last_kernels(tf_ctx* ctx, int32_t kernels[2]) {
+    if (!ctx || !kernels) return TF_ERR_INVALID_ARG;
+    kernels[0] = ctx->last_scan_kernel;
+    kernels[1] = ctx->last_attention_kernel;
+    return TF_OK;
+}
+
+tf_status tf_set_wait_limits(tf_ctx* ctx, int64_t max_polls, int64_t wait_cycles) {
+    if (!ctx) return TF_ERR_INVALID_ARG;
+    ctx->max_polls = max_polls < 0 ? -1 : max_polls;
+    ctx->wait_cycles = wait_cycles < 0 ? -1 : wait_cycles;
+    return TF_OK;
 }
 
 tf_status tf_set_attention_path(tf_ctx* ctx, int use_tensor_cores) {

@@ -132,6 +132,7 @@ cudaError_t launch_attention_simt(tf_ctx* ctx, const tf_shape& s, const tf_filte
     if (s.dtype == TF_BF16) attention_simt_kernel<__nv_bfloat16><<<grid, kSimtWarps * 32, 0, st>>>(ap);
     else                    attention_simt_kernel<float><<<grid, kSimtWarps * 32, 0, st>>>(ap);
     ctx->launches += 1;
+    ctx->last_attention_kernel = TF_KERNEL_ATTN_SIMT;
     return cudaGetLastError();
 }
 

@@ -26,11 +26,9 @@
 //
 // Every mbarrier wait is bounded by a cycle budget; on expiry the CTA records TF_ERR_TIMEOUT,
 // stops waiting, lets copies in flight land, releases its TMEM and exits.
-#include <cuda.h>
-
 #include <algorithm>
 
-#include "tf_common.cuh"
+#include "tf_ptx.cuh"
 
 namespace tf {
 namespace {
@@ -44,7 +42,6 @@ constexpr int kSoftmaxThreads = kQTiles * kTileM;
 constexpr int kThreads = kSoftmaxThreads + 128;   // third warpgroup: MMA warp, TMA warp, two idle warps
 constexpr int kMmaWarp = kSoftmaxThreads / 32, kTmaWarp = kMmaWarp + 1;
 constexpr uint32_t kTmemCols = 512;   // S0 | S1 | O0 | O1, 128 fp32 columns each
-constexpr long long kWaitCycles = 400000000ll;   // ~0.2 s at 2 GHz
 constexpr float kRescaleThreshold = 8.f;         // log2 units
 
 struct TcParams {
@@ -58,6 +55,7 @@ struct TcParams {
     int n_row_blocks;     // CTAs per (batch, query head)
     int heads_fastest;    // CTA order: 1 = all heads of the heaviest row block first, 0 = all row blocks of a head together
     int first_pair;       // row block the first CTA of a head takes: the last one expected to hold retained rows
+    long long wait_cycles;   // budget of one mbarrier wait
 };
 
 // Two ways of giving the two softmax groups of a CTA their work:
@@ -77,79 +75,11 @@ template <bool kSplit> struct Cfg {
     static constexpr int kSmemBytes = kOffBar + 256 + 1024;   // barriers + alignment slack
 };
 
-// ---- PTX wrappers -------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 // bounded wait; after the first expiry in this CTA nobody waits any more
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget_cycles,
                                           DevStatus* status, unsigned long long where) {
-    if (mbar_try_wait(bar, parity)) return;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (*abort_flag) return;
-        if (clock64() - t0 > kWaitCycles) {
-            *abort_flag = 1;
-            report_error(status, TF_ERR_TIMEOUT, where);
-            return;
-        }
-    }
+    mbar_wait_bounded(bar, parity, abort_flag, budget_cycles, status, where);
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-                 :: "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(dst_smem), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(addr), "r"(cols) : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                 : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-                 :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-                    "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-                    "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-                    "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -186,37 +116,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return d;
 }
 
-// Shared-memory operand descriptors (sm_100 format: version 1 at bit 46, swizzle mode at 61-63).
-// All operand blocks here are [rows][128 B] with the 128-byte swizzle; groups of 8 rows are 1024 B apart.
-//   K-major operand (Q, K, P): rows are M/N, the 128 B hold 64 consecutive K elements.
-//   MN-major operand (V):      rows are K (keys), the 128 B hold 64 consecutive N elements (dims);
-//                              the next 64 dims start one 16 KiB block later (leading byte offset).
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
-    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
-    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(kHalfBytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// instruction descriptor: D fp32, A/B bf16, M=128, N=128; bit 16 set = B is MN-major
-constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+// instruction descriptors: M=128, N=128; the P V product takes V as it lies in memory (MN-major)
+constexpr uint32_t kIdescQK = idesc_bf16(128, false, false);
+constexpr uint32_t kIdescPV = idesc_bf16(128, false, true);
 
 // byte offset of 16-byte chunk cc (0..15) of row r inside a two-block [128][64]+[128][64] operand
 __device__ __forceinline__ uint32_t swz(int r, int cc) {
     return (uint32_t)((cc >> 3) * kHalfBytes + r * 128 + (((cc & 7) ^ (r & 7)) << 4));
 }
 
-
-// D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-                 :: "r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
-}
 
 template <bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -244,7 +152,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         for (int i = 0; i < 2; ++i) { mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, kTileM); }
         mbar_init(bar_o, 1);
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_fence_init();
     }
     __syncwarp();
     if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
@@ -350,8 +258,8 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
                     // the first K and V tiles go out at once; the rest of the ring is filled once the Q rows are in shared
                     // memory (nothing can consume it earlier, and a ring's worth of arriving tiles keeps the gather's
                     // shared-memory stores waiting)
-                    if (q == 2) mbar_wait(bar_q, 0, abort_flag, p.status, 11);
-                    if (q >= kStages) mbar_wait(bar_empty + 8 * st, ((q / kStages) - 1) & 1, abort_flag, p.status, 10);
+                    if (q == 2) mbar_wait(bar_q, 0, abort_flag, p.wait_cycles, p.status, 11);
+                    if (q >= kStages) mbar_wait(bar_empty + 8 * st, ((q / kStages) - 1) & 1, abort_flag, p.wait_cycles, p.status, 10);
                     const uint32_t dst = sbase + kOffRing + st * kTileBytes;
                     const CUtensorMap* map = kv ? &mapV : &mapK;
                     mbar_expect_tx(bar_full + 8 * st, kTileBytes);
@@ -380,46 +288,46 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
                 const uint32_t vaddr = sbase + kOffRing + slot_of(j, 1) * kTileBytes;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, desc_mnmajor(vaddr + kk * 16 * 128), kIdescPV,
+                    mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, desc_mnmajor(vaddr + kk * 16 * 128, kHalfBytes), kIdescPV,
                            (!first || kk > 0) ? 1u : 0u);
             };
-            mbar_wait(bar_q, 0, abort_flag, p.status, 20);
+            mbar_wait(bar_q, 0, abort_flag, p.wait_cycles, p.status, 20);
             int done[kQTiles] = {0, 0};
             if constexpr (kSplit) {
                 // tile j belongs to group (j - J0) & 1; order: QK_0(J0), QK_1(J0+1), then per tile PV(j), QK(j+2)
                 for (int j = J0; j < min(J0 + 2, J1); ++j) {
-                    mbar_wait(bar_full + 8 * slot_of(j, 0), par_of(j, 0), abort_flag, p.status, 21);
+                    mbar_wait(bar_full + 8 * slot_of(j, 0), par_of(j, 0), abort_flag, p.wait_cycles, p.status, 21);
                     tc_fence_after();
                     issue_qk(j - J0, j);
                     mma_commit(bar_empty + 8 * slot_of(j, 0));
                 }
                 for (int j = J0; j < J1; ++j) {
                     const int i = (j - J0) & 1;
-                    mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.status, 22);
-                    mbar_wait(bar_p + 8 * i, done[i] & 1, abort_flag, p.status, 24 + i);
+                    mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.wait_cycles, p.status, 22);
+                    mbar_wait(bar_p + 8 * i, done[i] & 1, abort_flag, p.wait_cycles, p.status, 24 + i);
                     tc_fence_after();
                     issue_pv(i, j, done[i] == 0);
                     ++done[i];
                     mma_commit(bar_empty + 8 * slot_of(j, 1));
                     if (j + 2 < J1) {
-                        mbar_wait(bar_full + 8 * slot_of(j + 2, 0), par_of(j + 2, 0), abort_flag, p.status, 23);
+                        mbar_wait(bar_full + 8 * slot_of(j + 2, 0), par_of(j + 2, 0), abort_flag, p.wait_cycles, p.status, 23);
                         issue_qk(i, j + 2);
                         mma_commit(bar_empty + 8 * slot_of(j + 2, 0));
                     }
                 }
             } else {
-            mbar_wait(bar_full + 8 * slot_of(J0, 0), par_of(J0, 0), abort_flag, p.status, 21);
+            mbar_wait(bar_full + 8 * slot_of(J0, 0), par_of(J0, 0), abort_flag, p.wait_cycles, p.status, 21);
             tc_fence_after();
             for (int i = 0; i < kQTiles; ++i)
                 if (active(i, J0)) issue_qk(i, J0);
             mma_commit(bar_empty + 8 * slot_of(J0, 0));
             for (int j = J0; j < J1; ++j) {
-                mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.status, 22);
-                if (j + 1 < J1) mbar_wait(bar_full + 8 * slot_of(j + 1, 0), par_of(j + 1, 0), abort_flag, p.status, 23);
+                mbar_wait(bar_full + 8 * slot_of(j, 1), par_of(j, 1), abort_flag, p.wait_cycles, p.status, 22);
+                if (j + 1 < J1) mbar_wait(bar_full + 8 * slot_of(j + 1, 0), par_of(j + 1, 0), abort_flag, p.wait_cycles, p.status, 23);
 #pragma unroll
                 for (int i = 0; i < kQTiles; ++i) {
                     if (active(i, j)) {
-                        mbar_wait(bar_p + 8 * i, done[i] & 1, abort_flag, p.status, 24 + i);
+                        mbar_wait(bar_p + 8 * i, done[i] & 1, abort_flag, p.wait_cycles, p.status, 24 + i);
                         tc_fence_after();
                         issue_pv(i, j, done[i] == 0);
                         ++done[i];
@@ -468,7 +376,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         for (int j = jb[i]; j < je[i]; j += kStep) {
             const int c_it = (j - jb[i]) / kStep;
             const int j0 = j * kTileN;
-            mbar_wait(bar_s + 8 * i, c_it & 1, abort_flag, p.status, 30 + i);
+            mbar_wait(bar_s + 8 * i, c_it & 1, abort_flag, p.wait_cycles, p.status, 30 + i);
             __syncwarp();
             tc_fence_after();
             uint32_t sreg[128];
@@ -549,7 +457,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         if constexpr (kSplit) {
             // merge the two groups' partial results: both accumulators sit in the TMEM lanes of this row,
             // so each group finishes 64 of the 128 output columns
-            mbar_wait(bar_o, 0, abort_flag, p.status, 40);
+            mbar_wait(bar_o, 0, abort_flag, p.wait_cycles, p.status, 40);
             __syncwarp();
             tc_fence_after();
             float2* ml = reinterpret_cast<float2*>(smem + kOffRing);
@@ -597,7 +505,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
                         *reinterpret_cast<const uint4*>(smem + kOffQ + R * 256 + ((l16 ^ (R & 15)) << 4));
             }
         } else if (i < n_q) {
-            mbar_wait(bar_o, 0, abort_flag, p.status, 40);
+            mbar_wait(bar_o, 0, abort_flag, p.wait_cycles, p.status, 40);
             __syncwarp();
             tc_fence_after();
             const float inv = 1.f / l_run;
@@ -641,37 +549,9 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
-// ---- host side: tensor maps over the caller's K / V ----------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
+// ---- host side: tensor maps over the caller's K / V (two 64-column boxes of kTileN keys per tile) ---------
 bool make_kv_map(CUtensorMap* map, const void* base, const int64_t st[3], int B, int S, int H) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    // dims (fastest first): head_dim, head, token, batch
-    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)H, (cuuint64_t)S, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)st[2] * 2, (cuuint64_t)st[1] * 2,
-                                   (cuuint64_t)(st[0] > 0 ? st[0] : (int64_t)S * st[1]) * 2};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)kTileN, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return make_bshd_map(map, base, st, B, S, H, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kTileN, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // TF_KV_RETAINED: copy the retained tokens' K and V rows (all KV heads) to dense [B,S,Hkv,128] buffers,
@@ -748,10 +628,12 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         // releases 128 x 96, 168 -> 216 takes 256 x 48).  An inc only receives what a dec of the same CTA
         // released and waits for it without limit, so the trade must balance: refuse to launch a build that
         // does not start at 168 registers per thread.
+        // That is a defect of the build, not a property of the call: it is reported as an error of its own and
+        // never answered by running another kernel.
         cudaFuncAttributes fa{};
         if (cudaFuncGetAttributes(&fa, attention_tc_kernel<false>) != cudaSuccess || fa.numRegs != 168 ||
             cudaFuncGetAttributes(&fa, attention_tc_kernel<true>) != cudaSuccess || fa.numRegs != 168)
-            return cudaErrorNotSupported;
+            return cudaErrorInvalidDeviceFunction;
         attr_set = true;
     }
     TcParams tp{};
@@ -765,6 +647,7 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     tp.kept_idx = kept_idx; tp.n_kept = n_kept;
     tp.status = ctx->dev_status;
     tp.compact = compact ? 1 : 0;
+    tp.wait_cycles = ctx_wait_cycles(ctx);
     // The shared form needs enough CTAs to fill and balance the SMs (CTAs of one head differ in length by
     // the causal triangle); below that the split form, with twice as many CTAs of half the length, wins.
     // The number of retained rows is only known on the device: the ratio gives the expected count.
@@ -789,6 +672,7 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     if (split) e = launch_dependent(attention_tc_kernel<true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<true>::kSmemBytes, st, tp, mapK, mapV);
     else       e = launch_dependent(attention_tc_kernel<false>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     ctx->launches += 1;
+    ctx->last_attention_kernel = split ? TF_KERNEL_ATTN_TC_SPLIT : TF_KERNEL_ATTN_TC_SHARED;
     return e;
 }
 

@@ -108,13 +108,28 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 
 namespace tf {
 // Host-side bookkeeping of one scan scratch region (the first section of a workspace).
+// The region starts with two counter words {ticket, finished}: every CTA (or worker) of a scan launch draws its
+// work from `ticket`, and the last CTA to leave the kernel sets both words back to zero, so a launch always starts
+// counting at zero whatever happened to the launch before it (a wait that gave up, workers that stopped drawing).
 struct ScanScratch {
     void* ptr = nullptr;
-    size_t bytes = 0;               // bytes of the region the scan may use (cleared on first use)
+    size_t capacity = 0;            // bytes the owner of the region provides
+    size_t bytes = 0;               // layout key of the records cleared last (0: never cleared)
     unsigned int epoch = 0;         // tag of the latest launch
-    unsigned int ticket_base = 0;   // value of the ticket word before the next launch
     bool needs_clear = true;
 };
+constexpr size_t kScanCounterBytes = 256;   // {ticket, finished} + padding in front of the records
+
+// Drawn by one thread per CTA / worker after grid_dependency_wait().
+__device__ __forceinline__ unsigned int scan_draw_ticket(unsigned int* counters) { return atomicAdd(counters, 1u); }
+// Called by one thread per CTA when the CTA will draw no more tickets; n_ctas = gridDim.x.
+__device__ __forceinline__ void scan_leave(unsigned int* counters, unsigned int n_ctas) {
+    __threadfence();
+    if (atomicAdd(counters + 1, 1u) == n_ctas - 1u) {
+        atomicExch(counters, 0u);
+        atomicExch(counters + 1, 0u);
+    }
+}
 }  // namespace tf
 
 // The opaque context of include/tf.h.
@@ -129,6 +144,10 @@ struct tf_ctx {
     int scan_path;                 // tf_kv_stats: 0 = choose, 1 = plain CUDA-core kernel, 2 / 3 = Gram-matrix kernel, one tile per CTA / persistent
     int attention_form;            // tensor-core kernel: 0 = choose by grid size, 1 = shared K/V tiles, 2 = split K/V tiles
     long long launches;            // kernels launched through this context
+    int last_scan_kernel;          // TF_KERNEL_* of the latest similarity scan / attention launched through this context
+    int last_attention_kernel;
+    long long max_polls;           // bounded waits (tf_set_wait_limits): polls of a look-back record, < 0 = default
+    long long wait_cycles;         // ... and clock cycles of an mbarrier wait, < 0 = default
     // tf_layer_filter_host staging (owned, grown on demand)
     void* stage;
     size_t stage_bytes;
@@ -141,6 +160,13 @@ struct tf_ctx {
     cudaEvent_t ev[kHostEvents];
 };
 
+namespace tf {
+constexpr int kDefaultMaxPolls = 1 << 20;              // >= 32 ns apart plus an L2 round trip each: of the order of a second
+constexpr long long kDefaultWaitCycles = 1000000000ll; // ~0.5 s
+inline int ctx_max_polls(const tf_ctx* c) { return c->max_polls >= 0 ? (int)(c->max_polls > 0x7fffffff ? 0x7fffffff : c->max_polls) : kDefaultMaxPolls; }
+inline long long ctx_wait_cycles(const tf_ctx* c) { return c->wait_cycles >= 0 ? c->wait_cycles : kDefaultWaitCycles; }
+}  // namespace tf
+
 // ---- per-kernel launchers (defined in the .cu files, called by tf_api.cu) ----------------------
 namespace tf {
 
@@ -152,6 +178,12 @@ struct ScanPlan {            // how tf_kv_stats tiles a shape
     size_t bytes;            // scratch bytes (ticket word + records), 256-aligned
 };
 ScanPlan scan_plan(const tf_shape& s);
+size_t gram_scratch_bytes(const tf_shape& s);   // records of the Gram-matrix kernels (bf16), counters included
+// what tf_kv_stats may need for this shape whichever kernel it picks
+inline size_t scan_scratch_bytes(const tf_shape& s) {
+    const size_t a = scan_plan(s).bytes, b = s.dtype == TF_BF16 ? gram_scratch_bytes(s) : 0;
+    return a > b ? a : b;
+}
 
 cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                             const void* K, const void* V, float* sim_k, float* sim_v,
@@ -185,5 +217,7 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
                                 const int32_t* kept_idx, const int32_t* n_kept, void* O,
                                 void* kv_compact, cudaStream_t st);
 size_t kv_compact_bytes(const tf_shape& s);
+// marks the built-in scratch array of tf_kv_stats_static on `device` for clearing before its next use
+void static_scratch_invalidate(int device);
 
 }  // namespace tf

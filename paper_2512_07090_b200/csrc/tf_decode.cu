@@ -24,7 +24,8 @@ struct DecideParams {
     Strides3 ks, vs;
     const int32_t* pos;                 // [B] position of the current token
     int Hkv, anchor_mode, fuse_mode, warmup;
-    float gamma, var_eps, eta, target;
+    float gamma, var_eps, eta;
+    double target;                      // the target skip ratio, as the caller gave it
     int alg1_sign;
     float* sum_k; float* sum_v; long long* count;      // state
     float* tau; long long* steps; long long* skips;
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_decide_kernel(const Dec
             s += 0.f;
             // ratio and step in double, the threshold itself is an fp32 state word
             const double rho = steps > 0 ? (double)skips / (double)steps : 0.0;
-            const double delta = (double)p.eta * (p.alg1_sign ? ((double)p.target - rho) : (rho - (double)p.target));
+            const double delta = (double)p.eta * (p.alg1_sign ? (p.target - rho) : (rho - p.target));
             const float tau = tau_old + (float)delta;
             const bool decide = s > tau;              // false for NaN
             const bool skip = decide && t >= p.warmup;
@@ -418,7 +419,7 @@ cudaError_t launch_decode_step(tf_ctx* ctx, const tf_shape& s, const tf_filter_p
     dp.vs = {s.v_stride[0], s.v_stride[1], s.v_stride[2]};
     dp.pos = a.pos; dp.Hkv = s.n_kv_heads; dp.anchor_mode = p.anchor_mode; dp.fuse_mode = p.fuse_mode;
     dp.warmup = p.warmup_tokens; dp.gamma = p.gamma; dp.var_eps = p.var_eps > 0.f ? p.var_eps : 1e-8f;
-    dp.eta = a.eta; dp.target = (float)p.prune_ratio; dp.alg1_sign = a.alg1_sign;
+    dp.eta = a.eta; dp.target = p.prune_ratio; dp.alg1_sign = a.alg1_sign;
     dp.sum_k = a.state->sum_k; dp.sum_v = a.state->sum_v; dp.count = reinterpret_cast<long long*>(a.state->count);
     dp.tau = a.state->tau; dp.steps = reinterpret_cast<long long*>(a.state->steps);
     dp.skips = reinterpret_cast<long long*>(a.state->skips);

@@ -14,6 +14,7 @@
 // launches.  Tiles are handed out by an atomic ticket, chunk index slowest, so every record a
 // running tile waits for belongs to a tile that has itself started: the waits cannot deadlock,
 // and every wait is bounded anyway (on expiry the kernel records TF_ERR_TIMEOUT and goes on).
+// The last CTA to have drawn its ticket sets the counter back to zero for the next launch.
 //
 // Inside the CTA, 8 lanes share a token row (16 dims each, two 16-byte loads for bf16) and 16
 // such groups take consecutive runs of tokens; the groups' local sums are scanned through
@@ -44,7 +45,8 @@ struct ScanParams {
     const float* sum_k_in; const float* sum_v_in; const long long* count_in;
     float* sum_k_out; float* sum_v_out;
     float* sim_k; float* sim_v;
-    unsigned int* ticket; unsigned int ticket_base, epoch;
+    unsigned int* counters;   // {ticket, finished}: see ScanScratch
+    unsigned int epoch, n_tiles;
     uint4* agg_rec;      // [tile][128] packets, tile = chunk * n_chains + chain
     uint4* prefix_rec;   // [(chunk / kAnchorEvery) * n_chains + chain][128] packets
     DevStatus* status;
@@ -95,9 +97,13 @@ __global__ void __launch_bounds__(kScanThreads, 4) kv_stats_kernel(const ScanPar
     __shared__ unsigned int s_ticket;
 
     const int tid = threadIdx.x, g = tid >> 3, l = tid & 7;
-    if (tid == 0) s_ticket = atomicAdd(p.ticket, 1u) - p.ticket_base;
+    if (tid == 0) {
+        s_ticket = scan_draw_ticket(p.counters);
+        scan_leave(p.counters, gridDim.x);        // one ticket per CTA: this CTA draws no more
+    }
     __syncthreads();
     const unsigned int tile = s_ticket;
+    if (tile >= p.n_tiles) return;                // cannot happen while the counters are intact; never index records with it
     const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
     const int b = chain / p.H, h = chain % p.H;
     const int t0 = c * CH + g * TPG;
@@ -292,7 +298,7 @@ ScanPlan scan_plan(const tf_shape& s) {
     pl.n_chunks = (s.seq + pl.chunk_tokens - 1) / pl.chunk_tokens;
     const size_t tiles = (size_t)pl.n_chains * (size_t)pl.n_chunks;
     const size_t anchors = (size_t)pl.n_chains * (size_t)((pl.n_chunks + kAnchorEvery - 1) / kAnchorEvery);
-    pl.agg_offset = 256;                                                  // after the ticket word
+    pl.agg_offset = kScanCounterBytes;                                    // after the counter words
     pl.prefix_offset = pl.agg_offset + tiles * kHeadDim * sizeof(uint4);
     pl.bytes = pl.prefix_offset + anchors * kHeadDim * sizeof(uint4);
     pl.bytes = (pl.bytes + 255) / 256 * 256;
@@ -302,8 +308,12 @@ ScanPlan scan_plan(const tf_shape& s) {
 cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                             const void* K, const void* V, float* sim_k, float* sim_v,
                             const tf_carry* carry, ScanScratch* ws, cudaStream_t st) {
-    if (ctx->scan_path != 1 && kv_stats_gram_usable(s, p))
-        return launch_kv_stats_gram(ctx, s, p, K, V, sim_k, sim_v, carry, ws, st);
+    if (ctx->scan_path != 1 && kv_stats_gram_usable(s, p)) {
+        const cudaError_t e = launch_kv_stats_gram(ctx, s, p, K, V, sim_k, sim_v, carry, ws, st);
+        // an explicitly requested kernel is a requirement; the default falls back only when no tensor map can
+        // describe the caller's layout
+        if (e != cudaErrorNotSupported || ctx->scan_path >= 2) return e;
+    }
     if (ctx->scan_path >= 2) return cudaErrorNotSupported;
     const ScanPlan pl = scan_plan(s);
     const size_t tiles = (size_t)pl.n_chains * (size_t)pl.n_chunks;
@@ -313,13 +323,13 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
     // scratch region once when it is first used (and whenever the 32-bit epoch wraps).
     // The region is also cleared when its extent changes: another shape's layout may have put
     // other data where this shape keeps records.
+    if (ws->capacity < pl.bytes) return cudaErrorInvalidValue;
     if (ws->needs_clear || ws->bytes != pl.bytes || ws->epoch == 0xffffffffu) {
         cudaError_t e = cudaMemsetAsync(ws->ptr, 0, pl.bytes, st);
         if (e != cudaSuccess) return e;
         ws->needs_clear = false;
         ws->bytes = pl.bytes;
         ws->epoch = 0;
-        ws->ticket_base = 0;
     }
     ws->epoch += 1;
 
@@ -339,14 +349,13 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
     }
     sp.sim_k = sim_k; sp.sim_v = sim_v;
     char* base = static_cast<char*>(ws->ptr);
-    sp.ticket = reinterpret_cast<unsigned int*>(base);
-    sp.ticket_base = ws->ticket_base;
+    sp.counters = reinterpret_cast<unsigned int*>(base);
     sp.epoch = ws->epoch;
+    sp.n_tiles = (unsigned int)tiles;
     sp.agg_rec = reinterpret_cast<uint4*>(base + pl.agg_offset);
     sp.prefix_rec = reinterpret_cast<uint4*>(base + pl.prefix_offset);
     sp.status = ctx->dev_status;
-    sp.max_polls = 1 << 20;   // >= 32 ns apart plus an L2 round trip each: of the order of a second
-    ws->ticket_base += (unsigned int)tiles;   // the ticket word only ever counts up (mod 2^32)
+    sp.max_polls = ctx_max_polls(ctx);
 
     const dim3 grid((unsigned)tiles), block(kScanThreads);
     if (s.dtype == TF_BF16) {
@@ -357,7 +366,10 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
         else     kv_stats_kernel<float, false><<<grid, block, 0, st>>>(sp);
     }
     ctx->launches += 1;
-    return cudaGetLastError();
+    ctx->last_scan_kernel = TF_KERNEL_SCAN_PLAIN;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) ws->needs_clear = true;   // whatever the launch left behind is cleared before the next one
+    return e;
 }
 
 // ---------------------------------------------------------------------------------------------------

@@ -31,54 +31,9 @@ constexpr int kHalf = 128 * 128;               // one [128 rows][128 B] swizzled
 constexpr int kXBytes = 2 * kHalf;             // one tensor's tile
 constexpr int kBtBytes = 2 * 16 * 128;         // small B operand: [16 rows][128 elements], two 64-element blocks
 constexpr int kGramAnchorEvery = 4;             // a prefix record every 4th chunk: at most 4 aggregates + 1 prefix per look-back
-constexpr long long kGramWaitCycles = 1000000000ll;
 
-// ---- tcgen05 wrappers ---------------------------------------------------------------------------------
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(dst_smem), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                 : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory operand descriptors (sm_100: version 1 at bit 46, 128-byte swizzle at 61-63); 8-row groups 1024 B apart.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
-    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {   // next 64 MN elements one [128][128 B] block later
-    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(kHalf >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
 // instruction descriptors: D fp32, A/B bf16, M = 128
-constexpr uint32_t idesc(uint32_t n, bool a_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn ? (1u << 15) : 0u) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
+constexpr uint32_t idesc(uint32_t n, bool a_mn) { return idesc_bf16(n, a_mn, false); }
 constexpr uint32_t kIdescAgg = idesc(16, true);    // X^T Bt^T  (A = X taken MN-major: rows = dims)
 constexpr uint32_t kIdescU = idesc(16, false);     // X Bt^T
 
@@ -88,9 +43,9 @@ __device__ __forceinline__ uint32_t bt_off(int n, int k) {
 }
 __device__ __forceinline__ unsigned short bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
 
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevStatus* status,
-                                         unsigned long long where) {
-    return mbar_wait_bounded(bar, parity, abort_flag, kGramWaitCycles, status, where);
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget_cycles,
+                                         DevStatus* status, unsigned long long where) {
+    return mbar_wait_bounded(bar, parity, abort_flag, budget_cycles, status, where);
 }
 
 // ---- 8-byte record packets {value, tag}: one tensor per CTA --------------------------------------------
@@ -134,7 +89,10 @@ struct Gram1Params {
     unsigned int epoch;
     uint2* agg_rec[2]; uint2* prefix_rec[2];
     DevStatus* status;
-    int max_polls;
+    int max_polls;               // bounded waits: polls of one look-back packet ...
+    long long wait_cycles;       // ... and clock cycles of one mbarrier wait
+    unsigned int* counters;      // {ticket, finished}: see ScanScratch
+    unsigned int n_work;         // (tile, tensor) pairs
 };
 
 __global__ void __launch_bounds__(128, 6)
@@ -142,10 +100,16 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     extern __shared__ uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {   // the swizzled operand layout needs it; nothing has been started yet
-        if (threadIdx.x == 0) report_error(p.status, TF_ERR_TIMEOUT, 199);
+        if (threadIdx.x == 0) {
+            report_error(p.status, TF_ERR_TIMEOUT, 199);
+            grid_dependency_wait();
+            scan_draw_ticket(p.counters);
+            scan_leave(p.counters, gridDim.x);
+        }
         return;
     }
     const uint32_t bar_tma = sbase + kT1OffMisc, bar_mma = bar_tma + 8;
+    volatile unsigned int* s_ticket = reinterpret_cast<volatile unsigned int*>(smem + kT1OffMisc + 96);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kT1OffMisc + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kT1OffMisc + 24);
     float* red = reinterpret_cast<float*>(smem + kT1OffMisc + 32);     // [4 warps][2] block reduction / scan scratch
@@ -171,23 +135,37 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     const uint32_t tm_lane = tmem + ((uint32_t)(warp * 32) << 16);
     grid_dependency_wait();   // launched so that the set-up above overlaps the tail of the kernel before it on the stream
 
-    // Tiles go by block index (K and V of a tile side by side).  CTAs are started in index order, so the
-    // records a tile waits for belong to tiles started before it; should a scheduler ever break that order,
-    // the bounded waits turn the stall into TF_ERR_TIMEOUT instead of a hang.
-    const int x = blockIdx.x & 1;
-    const unsigned int tile = blockIdx.x >> 1;
+    // Work goes by ticket, chunk index slowest (K and V of a tile side by side): the records a tile waits for belong
+    // to tickets drawn before its own, by CTAs that are running, whatever order the CTAs were started in.
+    if (tid == 0) {
+        const unsigned int t = scan_draw_ticket(p.counters);
+        scan_leave(p.counters, gridDim.x);     // one ticket per CTA
+        *s_ticket = t;
+        if (t < p.n_work) {
+            const unsigned int tile0 = t >> 1;
+            const int c0 = (int)(tile0 / (unsigned)p.n_chains), chain0 = (int)(tile0 % (unsigned)p.n_chains);
+            const CUtensorMap* map = (t & 1) ? &mapV : &mapK;
+            mbar_expect_tx(bar_tma, kXBytes);
+            tma_load_4d(sbase + kT1OffX, map, bar_tma, 0, chain0 % p.H, c0 * kGT, chain0 / p.H);
+            tma_load_4d(sbase + kT1OffX + kHalf, map, bar_tma, 64, chain0 % p.H, c0 * kGT, chain0 / p.H);
+        }
+    }
+    __syncthreads();
+    const unsigned int ticket = *s_ticket;
+    if (ticket >= p.n_work) {                  // cannot happen while the counters are intact; never index records with it
+        tc_fence_before();
+        __syncthreads();
+        if (warp == 1) tmem_dealloc(tmem, kT1TmemCols);
+        return;
+    }
+    const int x = ticket & 1;
+    const unsigned int tile = ticket >> 1;
     const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
     const int b = chain / p.H, h = chain % p.H;
     const uint32_t xa = sbase + kT1OffX, bt = sbase + kT1OffBt;
     uint2* agg_rec = p.agg_rec[x];
     uint2* prefix_rec = p.prefix_rec[x];
 
-    if (tid == 0) {
-        const CUtensorMap* map = x ? &mapV : &mapK;
-        mbar_expect_tx(bar_tma, kXBytes);
-        tma_load_4d(xa, map, bar_tma, 0, h, c * kGT, b);
-        tma_load_4d(xa + kHalf, map, bar_tma, 64, h, c * kGT, b);
-    }
     // look-back requests go out while the tile is in flight
     const bool has_prev = c > 0;
     const int a0 = has_prev ? ((c - 1) / kGramAnchorEvery) * kGramAnchorEvery : 0;
@@ -203,18 +181,18 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     }
 
     uint32_t mma_phase = 0;
-    wait_bar(bar_tma, 0, abort_flag, p.status, 100);
+    wait_bar(bar_tma, 0, abort_flag, p.wait_cycles, p.status, 100);
 
     // ---- 1. column sums: (X^T Bt^T)[d][6] = sum_t X[t][d]; two interleaved accumulator chains ------------
     if (tid == 0) {
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)         // 16 tokens per step
-            mma_ss(tmem + 16 * (kk & 1), desc_mnmajor(xa + kk * 16 * 128),
+            mma_ss(tmem + 16 * (kk & 1), desc_mnmajor(xa + kk * 16 * 128, kHalf),
                    desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescAgg, kk > 1);
         mma_commit(bar_mma);
     }
-    wait_bar(bar_mma, mma_phase, abort_flag, p.status, 101); mma_phase ^= 1;
+    wait_bar(bar_mma, mma_phase, abort_flag, p.wait_cycles, p.status, 101); mma_phase ^= 1;
     tc_fence_after();
     float agg;
     {
@@ -261,7 +239,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
             }
             mma_commit(bar_mma);
         }
-        wait_bar(bar_mma, mma_phase, abort_flag, p.status, 102 + hh); mma_phase ^= 1;
+        wait_bar(bar_mma, mma_phase, abort_flag, p.wait_cycles, p.status, 102 + hh); mma_phase ^= 1;
         tc_fence_after();
 #pragma unroll
         for (int lc = 0; lc < 2; ++lc) {
@@ -313,7 +291,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
                    desc_kmajor(bt + (kk >> 2) * (16 * 128) + (kk & 3) * 32), kIdescU, kk > 1);
         mma_commit(bar_mma);
     }
-    wait_bar(bar_mma, mma_phase, abort_flag, p.status, 104); mma_phase ^= 1;
+    wait_bar(bar_mma, mma_phase, abort_flag, p.wait_cycles, p.status, 104); mma_phase ^= 1;
     tc_fence_after();
     float d;
     {
@@ -392,8 +370,7 @@ constexpr uint32_t kIdescG80 = idesc(80, false);
 constexpr int kPLookBack = kGramAnchorEvery - 1;                     // aggregates between a prefix record and a tile
 
 struct GramPParams {
-    Gram1Params g;
-    unsigned int* ticket; unsigned int ticket_base, n_tiles;        // n_tiles counts (tile, tensor) pairs
+    Gram1Params g;               // g.n_work counts (tile, tensor) pairs
 };
 
 // Eight products of one accumulation chain.  The operand descriptors differ only in the 14-bit address field of
@@ -417,8 +394,8 @@ __device__ __forceinline__ void mma_burst(std::integer_sequence<int, KK...>, uin
 }
 // mbarrier wait for the persistent kernel: the hardware may park the thread for up to the hinted time per try, and
 // the clock and the abort flag are looked at once per 32 tries, so a waiting warp costs few issue slots
-__device__ __forceinline__ bool wait_bar_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevStatus* status,
-                                                unsigned long long where) {
+__device__ __forceinline__ bool wait_bar_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget_cycles,
+                                                DevStatus* status, unsigned long long where) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -430,7 +407,7 @@ __device__ __forceinline__ bool wait_bar_parked(uint32_t bar, uint32_t parity, v
             if (ok) return true;
         }
         if (*abort_flag) return false;
-        if (clock64() - t0 > kGramWaitCycles) {
+        if (clock64() - t0 > budget_cycles) {
             *abort_flag = 1;
             report_error(status, TF_ERR_TIMEOUT, where);
             return false;
@@ -442,10 +419,6 @@ __device__ __forceinline__ void worker_sync(int w) { asm volatile("bar.sync %0, 
 __device__ __forceinline__ uint32_t pbt_off(int n, int k) {
     return (uint32_t)((k >> 6) * kPBlock + kHalf + n * 128 + ((((k & 63) >> 3) ^ (n & 7)) << 4) + (k & 7) * 2);
 }
-__device__ __forceinline__ uint64_t pdesc_mnmajor(uint32_t addr) {   // next 64 MN elements one block later
-    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(kPBlock >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
 
 __global__ void __launch_bounds__(kPThreads, 1)
 kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CUtensorMap mapK,
@@ -454,7 +427,11 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
     const Gram1Params& p = pp.g;
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {
-        if (threadIdx.x == 0) report_error(p.status, TF_ERR_TIMEOUT, 299);
+        if (threadIdx.x == 0) {
+            report_error(p.status, TF_ERR_TIMEOUT, 299);
+            grid_dependency_wait();
+            scan_leave(p.counters, gridDim.x);
+        }
         return;
     }
     const int tid = threadIdx.x & 127, w = threadIdx.x >> 7, warp = tid >> 5, lane = tid & 31;
@@ -490,7 +467,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
     const uint32_t tmem = *tmem_slot;
     const uint32_t tm_g = tmem + 80u * w, tm_s = tm_g + 64u;                       // G half / small product
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    // operand descriptor words (see desc_kmajor / pdesc_mnmajor): address field of this worker's tile, the two
+    // operand descriptor words (see desc_kmajor / desc_mnmajor): address field of this worker's tile, the two
     // leading-dimension fields, and the high word (8-row groups 1024 B apart, version 1, 128-byte swizzle)
     const uint32_t x_lo = (xa & 0x3ffffu) >> 4;
     constexpr uint32_t dlo_k = 1u << 16, dlo_mn = (uint32_t)(kPBlock >> 4) << 16;
@@ -514,8 +491,8 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         tma_load_4d(xa + kPBlock, map, bar_tma, 64, (int)h, (int)c * kGT, (int)b);
     };
     auto draw = [&]() -> unsigned int {
-        const unsigned int t = atomicAdd(pp.ticket, 1u) - pp.ticket_base;
-        return t < pp.n_tiles ? t : kPNoTile;
+        const unsigned int t = scan_draw_ticket(p.counters);
+        return t < p.n_work ? t : kPNoTile;
     };
 
     grid_dependency_wait();   // the set-up above overlaps the tail of the kernel before this one on the stream
@@ -533,7 +510,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         if (tid == 0) t_next = draw();                       // the answer is needed only when this tile's products are done
         const long long cnt0 = p.count_in ? p.count_in[b] : 0ll;
 
-        wait_bar_parked(bar_tma, tile_phase, abort_flag, p.status, 200);
+        wait_bar_parked(bar_tma, tile_phase, abort_flag, p.wait_cycles, p.status, 200);
 
         // ---- X^T 1 (columns 64-79) and columns 0-63 of G, issued together ------------------------------------
         if (tid == 0) {
@@ -556,7 +533,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
                 if (a0 + u < c) afirst[u] = ld_packet2(arec + u * astride);
         }
 
-        wait_bar_parked(bar_small, tile_phase, abort_flag, p.status, 201);
+        wait_bar_parked(bar_small, tile_phase, abort_flag, p.wait_cycles, p.status, 201);
         tile_phase ^= 1;
         tc_fence_after();
         float agg;
@@ -619,7 +596,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
                 }
             }
         };
-        wait_bar_parked(bar_g, 0, abort_flag, p.status, 202);
+        wait_bar_parked(bar_g, 0, abort_flag, p.wait_cycles, p.status, 202);
         tc_fence_after();
         add_half(0);
         fence_proxy_async();
@@ -632,7 +609,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             mma_burst<kPBlock, false>(k8, tm_g, x_lo | dlo_k, dhi, x_lo + (64 * 128 >> 4) | dlo_k, dhi, kIdescG80);
             mma_commit(bar_g);
         }
-        wait_bar_parked(bar_g, 1, abort_flag, p.status, 203);
+        wait_bar_parked(bar_g, 1, abort_flag, p.wait_cycles, p.status, 203);
         tc_fence_after();
         // every product that reads this tile has completed: the next one may land on it
         if (tid == 0) announce_and_load(*abort_flag ? kPNoTile : t_next);
@@ -687,6 +664,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         __syncthreads();
     }
     if (threadIdx.x < 32) tmem_dealloc(tmem, kPTmemCols);
+    if (threadIdx.x == 0) scan_leave(p.counters, gridDim.x);   // every worker of this CTA has stopped drawing
 }
 
 }  // namespace
@@ -695,36 +673,51 @@ bool kv_stats_gram_usable(const tf_shape& s, const tf_filter_params& p) {
     return s.dtype == TF_BF16 && p.anchor_mode != TF_ANCHOR_EMA;
 }
 
+namespace {
+// scratch: the counter words, then per tensor one 1 KiB record (128 packets of 8 bytes) per tile and one per
+// kGramAnchorEvery-th chunk of a chain
+struct GramLayout { size_t tiles, anchors, agg_offset, prefix_offset, bytes; int n_chains, n_chunks; };
+GramLayout gram_layout(const tf_shape& s) {
+    GramLayout g{};
+    g.n_chains = s.batch * s.n_kv_heads;
+    g.n_chunks = (s.seq + kGT - 1) / kGT;
+    g.tiles = (size_t)g.n_chains * (size_t)g.n_chunks;
+    g.anchors = (size_t)g.n_chains * (size_t)((g.n_chunks + kGramAnchorEvery - 1) / kGramAnchorEvery);
+    const size_t rec = kHeadDim * sizeof(uint2);
+    g.agg_offset = kScanCounterBytes;
+    g.prefix_offset = g.agg_offset + 2 * g.tiles * rec;
+    g.bytes = (g.prefix_offset + 2 * g.anchors * rec + 255) / 256 * 256;
+    return g;
+}
+}  // namespace
+
+size_t gram_scratch_bytes(const tf_shape& s) { return gram_layout(s).bytes; }
+
 cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                                  const void* K, const void* V, float* sim_k, float* sim_v,
                                  const tf_carry* carry, ScanScratch* ws, cudaStream_t st) {
-    const int n_chains = s.batch * s.n_kv_heads;
-    const int n_chunks = (s.seq + kGT - 1) / kGT;
-    const size_t tiles = (size_t)n_chains * (size_t)n_chunks;
+    const GramLayout gl = gram_layout(s);
+    const size_t tiles = gl.tiles;
     if (tiles == 0) return cudaSuccess;
     if (2 * tiles > 0x7fffffffu) return cudaErrorInvalidValue;
-    // scratch: per tensor, one 1 KiB record (128 packets of 8 bytes) per tile and one per 8th chunk of a chain
-    const size_t anchors = (size_t)n_chains * (size_t)((n_chunks + kGramAnchorEvery - 1) / kGramAnchorEvery);
-    const size_t rec = kHeadDim * sizeof(uint2);
-    const size_t agg_offset = 256, prefix_offset = agg_offset + 2 * tiles * rec;
-    // (the low bit distinguishes this kernel's record layout from the plain kernel's, which may share the scratch)
-    const size_t bytes = ((prefix_offset + 2 * anchors * rec + 255) / 256 * 256) | 1;
-    if (ws->needs_clear || ws->bytes != bytes || ws->epoch == 0xffffffffu) {
-        cudaError_t e = cudaMemsetAsync(ws->ptr, 0, bytes & ~(size_t)1, st);
-        if (e != cudaSuccess) return e;
-        ws->needs_clear = false;
-        ws->bytes = bytes;
-        ws->epoch = 0;
-        ws->ticket_base = 0;
-    }
-    ws->epoch += 1;
-
+    if (ws->capacity < gl.bytes) return cudaErrorInvalidValue;
     CUtensorMap mk, mv;
     if (!make_bshd_map(&mk, K, s.k_stride, s.batch, s.seq, s.n_kv_heads, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kGT,
                        CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_bshd_map(&mv, V, s.v_stride, s.batch, s.seq, s.n_kv_heads, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kGT,
                        CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorNotSupported;
+    // (the low bit of the layout key distinguishes this record layout from the plain kernel's, which may share the scratch)
+    const size_t key = gl.bytes | 1;
+    if (ws->needs_clear || ws->bytes != key || ws->epoch == 0xffffffffu) {
+        cudaError_t e = cudaMemsetAsync(ws->ptr, 0, gl.bytes, st);
+        if (e != cudaSuccess) return e;
+        ws->needs_clear = false;
+        ws->bytes = key;
+        ws->epoch = 0;
+    }
+    ws->epoch += 1;
+
     static bool attr_set_dev[kDeviceFlagSlots] = {};      // function attributes are per device
     bool& attr_set = attr_set_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
     if (!attr_set) {
@@ -733,7 +726,7 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
         attr_set = true;
     }
     Gram1Params gp{};
-    gp.S = s.seq; gp.H = s.n_kv_heads; gp.n_chains = n_chains; gp.n_chunks = n_chunks;
+    gp.S = s.seq; gp.H = s.n_kv_heads; gp.n_chains = gl.n_chains; gp.n_chunks = gl.n_chunks;
     gp.incl = (p.anchor_mode == TF_ANCHOR_INCL_MEAN);
     if (carry) {
         gp.sum_in[0] = carry->sum_k_in; gp.sum_in[1] = carry->sum_v_in;
@@ -743,38 +736,42 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     gp.sim[0] = sim_k; gp.sim[1] = sim_v;
     char* base = static_cast<char*>(ws->ptr);
     gp.epoch = ws->epoch;
+    const size_t rec = kHeadDim * sizeof(uint2);
     for (int x = 0; x < 2; ++x) {
-        gp.agg_rec[x] = reinterpret_cast<uint2*>(base + agg_offset + x * tiles * rec);
-        gp.prefix_rec[x] = reinterpret_cast<uint2*>(base + prefix_offset + x * anchors * rec);
+        gp.agg_rec[x] = reinterpret_cast<uint2*>(base + gl.agg_offset + x * tiles * rec);
+        gp.prefix_rec[x] = reinterpret_cast<uint2*>(base + gl.prefix_offset + x * gl.anchors * rec);
     }
     gp.status = ctx->dev_status;
-    gp.max_polls = 1 << 20;
+    gp.max_polls = ctx_max_polls(ctx);
+    gp.wait_cycles = ctx_wait_cycles(ctx);
+    gp.counters = reinterpret_cast<unsigned int*>(base);
+    gp.n_work = (unsigned int)(2 * tiles);
     int sms = 148;
     { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
     // the persistent form pays its set-up once per SM and wins once every worker sees several tiles (measured
     // cross-over between 2.3 and 11.5 tiles per worker); below that the one-tile-per-CTA form starts sooner
     const bool persistent = ctx->scan_path == 3 || (ctx->scan_path == 0 && 2 * tiles >= (size_t)4 * sms * kPWorkers);
+    cudaError_t e;
     if (persistent) {
         static bool attr_set_p_dev[kDeviceFlagSlots] = {};
         bool& attr_set_p = attr_set_p_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
         if (!attr_set_p) {
-            cudaError_t e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
+            e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
             if (e != cudaSuccess) return e;
             attr_set_p = true;
         }
-        const unsigned int n_work = (unsigned int)(2 * tiles);
-        const unsigned int grid = std::min<unsigned int>((unsigned int)sms, (n_work + kPWorkers - 1) / kPWorkers);
+        const unsigned int grid = std::min<unsigned int>((unsigned int)sms, (gp.n_work + kPWorkers - 1) / kPWorkers);
         GramPParams pp{};
         pp.g = gp;
-        pp.ticket = reinterpret_cast<unsigned int*>(base);
-        pp.ticket_base = ws->ticket_base;
-        pp.n_tiles = n_work;
-        ws->ticket_base += n_work + grid * kPWorkers;      // every worker draws once past the end
-        ctx->launches += 1;
-        return launch_dependent(kv_stats_gram_persistent_kernel, dim3(grid), dim3(kPThreads), kPSmem, st, pp, mk, mv);
+        e = launch_dependent(kv_stats_gram_persistent_kernel, dim3(grid), dim3(kPThreads), kPSmem, st, pp, mk, mv);
+        ctx->last_scan_kernel = TF_KERNEL_SCAN_GRAM_PERSISTENT;
+    } else {
+        e = launch_dependent(kv_stats_gram1_kernel, dim3(gp.n_work), dim3(128), kT1Smem, st, gp, mk, mv);
+        ctx->last_scan_kernel = TF_KERNEL_SCAN_GRAM_TILE;
     }
     ctx->launches += 1;
-    return launch_dependent(kv_stats_gram1_kernel, dim3((unsigned)(2 * tiles)), dim3(128), kT1Smem, st, gp, mk, mv);
+    if (e != cudaSuccess) ws->needs_clear = true;   // whatever the launch left behind is cleared before the next one
+    return e;
 }
 
 }  // namespace tf

@@ -55,7 +55,7 @@ extern "C" tf_status tf_kv_stats_static(tf_ctx* ctx, const tf_shape* shape, cons
     if ((reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V)) & 15u) return TF_ERR_UNSUPPORTED;
 
     // the whole point of this entry: a shape whose records do not fit is refused, never grown
-    if (scan_plan(*shape).bytes > kStaticScratchBytes) return TF_ERR_WORKSPACE;
+    if (scan_scratch_bytes(*shape) > kStaticScratchBytes) return TF_ERR_WORKSPACE;
 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TF_ERR_CUDA;
@@ -71,12 +71,20 @@ extern "C" tf_status tf_kv_stats_static(tf_ctx* ctx, const tf_shape* shape, cons
         }
         slot.scan = ScanScratch();
         slot.scan.ptr = ptr;      // needs_clear is set: the first launch zeroes the record region
+        slot.scan.capacity = kStaticScratchBytes;
         slot.ready = true;
     }
     tf_ctx local{};               // without a context nothing records device-side conditions
     local.device = dev;
+    local.max_polls = local.wait_cycles = -1;
     tf_ctx* use = ctx ? ctx : &local;
     cudaError_t e = launch_kv_stats(use, *shape, *params, K, V, sim_k, sim_v, carry, &slot.scan,
                                     static_cast<cudaStream_t>(stream));
-    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    return e == cudaSuccess ? TF_OK : (e == cudaErrorNotSupported ? TF_ERR_UNSUPPORTED : TF_ERR_CUDA);
+}
+
+void tf::static_scratch_invalidate(int device) {
+    if (device < 0 || device >= kMaxDevices) return;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_slots[device].scan.needs_clear = true;
 }

@@ -33,6 +33,7 @@ def test_kv_stats_matches_oracle(dtype, B, S, Hkv, scan_path):
     g.ctx.tf_set_scan_path(scan_path)
     g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
     g.status_ok()
+    assert g.ctx.tf_last_kernels()[0] == scan_path          # the kernel asked for is the kernel that ran
     _, kn, vn = oracle_inputs(q, k, v)
     assert np.abs(to_np(g.sim_k) - oracle.anchor_similarity(kn)).max() < SCORE_ATOL
     assert np.abs(to_np(g.sim_v) - oracle.anchor_similarity(vn)).max() < SCORE_ATOL
@@ -99,9 +100,12 @@ def test_kv_stats_head_major_layout_and_carry(scan_path):
     g = Gpu(q, kt, vt)
     g.ctx.tf_set_scan_path(scan_path)
     g.ctx.tf_kv_stats(g.shape, g.params, kt, vt, g.sim_k, g.sim_v)
+    g.status_ok()
     _, kn, vn = oracle_inputs(q, k, v)
     ref_k, sum_k = oracle.anchor_similarity(kn, want_sum_out=True)
+    ref_v, sum_v = oracle.anchor_similarity(vn, want_sum_out=True)
     assert np.abs(to_np(g.sim_k) - ref_k).max() < SCORE_ATOL
+    assert np.abs(to_np(g.sim_v) - ref_v).max() < SCORE_ATOL
     g.close()
     # chained halves
     h = S // 2
@@ -117,9 +121,13 @@ def test_kv_stats_head_major_layout_and_carry(scan_path):
     c2 = tfb.tf_carry(sk.data_ptr(), sv.data_ptr(), cnt.data_ptr(), sk2.data_ptr(), sv2.data_ptr())
     g2.ctx.tf_kv_stats(g2.shape, g2.params, k[:, h:], v[:, h:], g2.sim_k, g2.sim_v, c2)
     g2.status_ok()
+    g1.status_ok()
     both = np.concatenate([to_np(g1.sim_k), to_np(g2.sim_k)], 1)
     assert np.abs(both - ref_k).max() < SCORE_ATOL
+    both_v = np.concatenate([to_np(g1.sim_v), to_np(g2.sim_v)], 1)
+    assert np.abs(both_v - ref_v).max() < SCORE_ATOL
     assert np.abs(to_np(sk2) - sum_k).max() < 1e-3 * max(1.0, np.abs(sum_k).max())
+    assert np.abs(to_np(sv2) - sum_v).max() < 1e-3 * max(1.0, np.abs(sum_v).max())
     g1.close(); g2.close()
 
 
@@ -230,11 +238,25 @@ def test_pruned_attention_matches_oracle(dtype, tensor_cores, B, S, Hq, Hkv, win
     nk = torch.from_numpy(ref["n_kept"]).to(DEV)
     g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
     g.status_ok()
+    _assert_attention_kernel(g.ctx, dtype, tensor_cores)
     o = to_np(g.O)
     assert np.isfinite(o).all()
     assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
     assert np.all(o[ref["keep_mask"] == 0] == 0.0)
     g.close()
+
+
+def _assert_attention_kernel(ctx, dtype, path):
+    """The kernel that ran is the one the path names: 0 CUDA cores, 2 / 3 the tensor-core kernel's shared / split
+    form (a build whose tensor-core kernel cannot be launched fails the call instead of running on CUDA cores),
+    1 the tensor-core kernel in either form."""
+    ran = ctx.tf_last_kernels()[1]
+    if dtype != torch.bfloat16 or path == 0:
+        assert ran == tfb.TF_KERNEL_ATTN_SIMT
+    elif path == 1:
+        assert ran in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT)
+    else:
+        assert ran == {2: tfb.TF_KERNEL_ATTN_TC_SHARED, 3: tfb.TF_KERNEL_ATTN_TC_SPLIT}[path]
 
 
 @pytest.mark.parametrize("dtype,path", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 0), (torch.float32, 0)])
@@ -254,6 +276,7 @@ def test_pruned_attention_retained_keys_only(dtype, path, B, S, Hq, Hkv, window,
     nk = torch.from_numpy(ref["n_kept"]).to(DEV)
     g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
     g.status_ok()
+    _assert_attention_kernel(g.ctx, dtype, path)
     o = to_np(g.O)
     assert np.isfinite(o).all()
     assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
@@ -446,6 +469,106 @@ def test_device_rejects_bad_arguments_without_launching():
     g.close()
 
 
+# ------------------------------------------------------------------------------- device status record
+def test_nan_score_is_reported_counted_and_cleared():
+    """A NaN similarity makes the fused score NaN: tf_get_status returns TF_ERR_NAN_SCORE with the count of NaN
+    scores, the selection never prunes such a token, and tf_clear_status resets the record."""
+    B, S, H = 2, 300, 4
+    rng = np.random.default_rng(7)
+    ck = rng.uniform(-0.2, 0.8, (B, S, H)).astype(np.float32)
+    cv = rng.uniform(-0.2, 0.8, (B, S, H)).astype(np.float32)
+    ck[0, 17, 1] = np.nan; cv[1, 200, 0] = np.nan; ck[1, 250, 3] = np.nan
+    q = torch.zeros(B, S, H, 128, dtype=torch.bfloat16, device=DEV)
+    g = Gpu(q, q, q, prune_ratio=0.5, warmup_tokens=0)
+    g.ctx.tf_score_fuse(g.shape, g.params, torch.from_numpy(ck).to(DEV), torch.from_numpy(cv).to(DEV), g.score)
+    code, det = g.ctx.tf_get_status()
+    assert code == tfb.TF_ERR_NAN_SCORE and det["code"] == tfb.TF_ERR_NAN_SCORE
+    assert det["nan_count"] == 3
+    assert det["where"] in (0 * S + 17, 1 * S + 200, 1 * S + 250)      # the token index of the first one seen
+    sc = to_np(g.score)
+    assert np.isnan(sc[0, 17]) and np.isnan(sc[1, 200]) and np.isnan(sc[1, 250]) and np.isnan(sc).sum() == 3
+    g.ctx.tf_select(g.shape, g.params, g.score, g.keep, g.idx, g.nk, g.theta)
+    keep = g.keep.cpu().numpy()
+    assert keep[0, 17] == 1 and keep[1, 200] == 1 and keep[1, 250] == 1
+    ref = oracle.select(sc.astype(np.float64), 0.5, 0)
+    assert np.array_equal(keep, ref["keep_mask"]) and list(ref["n_nan"]) == [1, 2]
+    g.ctx.tf_clear_status()
+    code, det = g.ctx.tf_get_status()
+    assert code == tfb.TF_OK and det["nan_count"] == 0 and det["code"] == 0
+    g.close()
+
+
+def test_bounded_wait_that_runs_out_is_reported_and_the_context_recovers():
+    """Two chunks of one sequence and one head, on the Gram kernel that takes one tile per CTA, with the look-back
+    limit set to 0 polls.  The CTAs of the second chunk ask for the first chunk's records as soon as they start,
+    long before the first chunk's tile has even arrived from memory, so that look finds nothing and, with no polls
+    allowed, the wait runs out: the kernel finishes (no hang, no trap), tf_get_status returns TF_ERR_TIMEOUT with the
+    tile that gave up, and after tf_clear_status and the default limits the same context gives the right answer."""
+    q, k, v = _qkv(1, 256, 1, 1, torch.bfloat16, seed=3)
+    g = Gpu(q, k, v)
+    _, kn, vn = oracle_inputs(q, k, v)
+    ref_k, ref_v = oracle.anchor_similarity(kn), oracle.anchor_similarity(vn)
+    g.ctx.tf_set_scan_path(2)
+    g.ctx.tf_set_wait_limits(max_polls=0)
+    g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    code, det = g.ctx.tf_get_status()
+    assert code == tfb.TF_ERR_TIMEOUT and det["code"] == tfb.TF_ERR_TIMEOUT
+    assert det["where"] == 1                                   # chunk 1 of chain 0 is the tile that waited
+    assert torch.isfinite(g.sim_k).all()                       # the kernel ran to its end
+    assert np.abs(to_np(g.sim_k)[:, :128] - ref_k[:, :128]).max() < SCORE_ATOL   # chunk 0 waits for nobody
+    g.ctx.tf_clear_status()
+    g.ctx.tf_set_wait_limits()                                 # defaults again
+    for path in (2, 3, 1):
+        g.sim_k.fill_(float("nan")); g.sim_v.fill_(float("nan"))
+        g.ctx.tf_set_scan_path(path)
+        g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+        g.status_ok()
+        assert np.abs(to_np(g.sim_k) - ref_k).max() < SCORE_ATOL
+        assert np.abs(to_np(g.sim_v) - ref_v).max() < SCORE_ATOL
+    g.close()
+
+
+@pytest.mark.parametrize("scan_path", [1, 3])
+def test_zero_poll_limit_never_hangs_and_the_next_launch_is_clean(scan_path):
+    """The same zero-poll limit on the two ticketed kernels whose look-back happens later in a tile's life (whether a
+    record is already there is then a matter of timing): whatever the status says, the call returns, and the next
+    launch with default limits is right -- the counters a launch draws its work from start at zero again."""
+    q, k, v = _qkv(2, 1500, 3, 3, torch.bfloat16, seed=4)
+    g = Gpu(q, k, v)
+    _, kn, vn = oracle_inputs(q, k, v)
+    g.ctx.tf_set_scan_path(scan_path)
+    g.ctx.tf_set_wait_limits(max_polls=0)
+    for _ in range(2):
+        g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    code, _ = g.ctx.tf_get_status()
+    assert code in (tfb.TF_OK, tfb.TF_ERR_TIMEOUT)
+    g.ctx.tf_clear_status()
+    g.ctx.tf_set_wait_limits()
+    g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    g.status_ok()
+    assert np.abs(to_np(g.sim_k) - oracle.anchor_similarity(kn)).max() < SCORE_ATOL
+    assert np.abs(to_np(g.sim_v) - oracle.anchor_similarity(vn)).max() < SCORE_ATOL
+    g.close()
+
+
+def test_requested_kernel_that_cannot_take_the_call_is_an_error_not_a_fallback():
+    q, k, v = _qkv(1, 200, 2, 2, torch.float32)
+    g = Gpu(q, k, v)
+    for path in (2, 3):                                        # the Gram kernels take bf16 only
+        g.ctx.tf_set_scan_path(path)
+        with pytest.raises(tfb.TokenFilterError) as e:
+            g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+        assert e.value.code == tfb.TF_ERR_UNSUPPORTED
+    g.close()
+    q, k, v = _qkv(1, 200, 2, 2, torch.bfloat16)
+    g = Gpu(q, k, v, anchor_mode=tfb.TF_ANCHOR_EMA)
+    g.ctx.tf_set_scan_path(2)                                  # ... and running-sum anchors only
+    with pytest.raises(tfb.TokenFilterError) as e:
+        g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
+    assert e.value.code == tfb.TF_ERR_UNSUPPORTED
+    g.close()
+
+
 # ------------------------------------------------------------------------------- online decode step
 @pytest.mark.parametrize("dtype,mode,window,S0,T,Hq,Hkv",
                          [(torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0, 70, 90, 8, 2), (torch.float32, tfb.TF_ANCHOR_PAST_MEAN, 40, 70, 90, 8, 2),
@@ -455,9 +578,12 @@ def test_device_rejects_bad_arguments_without_launching():
                           (torch.bfloat16, tfb.TF_ANCHOR_PAST_MEAN, 0, 1100, 24, 6, 3)])
 def test_decode_steps_match_oracle(dtype, mode, window, S0, T, Hq, Hkv):
     """A prefill of 70 tokens seeds the anchors through tf_kv_stats' carry; then 90 decode steps run in
-    lockstep with the oracle: scores within 1e-5, thresholds within 1e-6, skip decisions equal unless the
-    score is within 1e-5 of the threshold (then the oracle's state is forced on so the runs stay comparable),
-    outputs within the attention tolerance; skipped rows are zero."""
+    lockstep with the oracle: scores within 1e-5, skip decisions equal unless the score is within 1e-5 of
+    the threshold (then the oracle's counters are forced on so the runs stay comparable), outputs within the
+    attention tolerance; skipped rows are zero.  The oracle is fp64 throughout; the library's threshold is an
+    fp32 state word (tf_decode_state.tau) and its step size an fp32 argument, so the oracle is given the same
+    fp32 value of eta, and after n updates the two thresholds may differ by n roundings of an fp32 sum:
+    |tau_gpu - tau_oracle| <= n * 2^-23 * max(1, |tau|)  (one rounding of the step, one of the sum, per update)."""
     B = 2
     S = S0 + T
     q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=123, dup=0.4)
@@ -484,13 +610,16 @@ def test_decode_steps_match_oracle(dtype, mode, window, S0, T, Hq, Hkv):
     shape.o_stride[:] = [O.stride(0), 0, O.stride(1)]
     score = torch.empty(B, device=DEV); skip = torch.empty(B, dtype=torch.uint8, device=DEV)
     near, n_skips = 0, 0
+    eta = float(np.float32(0.05))         # the value the C-ABI's float argument carries
     for t in range(S0, S):
         pos = torch.full((B,), t, dtype=torch.int32, device=DEV)
-        ctx.tf_decode_step(shape, params, 0.05, q[:, t], k, v, pos, st, O, score, skip)
-        ref = oracle.decode_step(ost, qn[:, t], kn, vn, np.full(B, t), target_ratio=0.25, eta=0.05, warmup_tokens=4,
+        ctx.tf_decode_step(shape, params, eta, q[:, t], k, v, pos, st, O, score, skip)
+        ref = oracle.decode_step(ost, qn[:, t], kn, vn, np.full(B, t), target_ratio=0.25, eta=eta, warmup_tokens=4,
                                  anchor_mode=mode, gamma=0.9, window=window)
         assert np.abs(to_np(score) - ref["score"]).max() < SCORE_ATOL
-        assert np.abs(to_np(st.tau) - ref["tau"]).max() < 1e-6
+        n_upd = t - S0 + 1
+        tau_gpu = st.tau.cpu().numpy().astype(np.float64)
+        assert np.abs(tau_gpu - ref["tau"]).max() <= n_upd * 2.0 ** -23 * max(1.0, np.abs(ref["tau"]).max())
         g_skip = skip.cpu().numpy()
         for b in range(B):
             if g_skip[b] != ref["skip"][b]:

@@ -5,14 +5,16 @@ leave the device heap to a framework's allocator, cannot provide the scratch tf_
 tf_kv_stats_static keeps that scratch in an array built into the library.  Here it is called
 through the C-ABI twice in a row (different inputs and shapes, so the second call finds the first
 call's records in the shared array) and each result is compared with tf_kv_stats on a caller-owned
-workspace.  The file sorts last so that a run that stops at the first failure has already gone
+workspace and with the fp64 oracle on the same bytes.  The file sorts last so that a run that stops at the first failure has already gone
 through every other test.
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2512_07090_b200 import binding as tfb, workloads as W
 from parity import SCORE_ATOL
 
@@ -40,6 +42,11 @@ def _both(ctx, B, S, H, dtype, seed, check_free=True, **params):
     assert not torch.isnan(out_k).any() and not torch.isnan(out_v).any()
     assert (out_k - ref_k).abs().max().item() < SCORE_ATOL
     assert (out_v - ref_v).abs().max().item() < SCORE_ATOL
+    mode, gamma = params.get("anchor_mode", tfb.TF_ANCHOR_PAST_MEAN), params.get("gamma", 0.9)
+    want_k = oracle.anchor_similarity(k.float().cpu().numpy(), mode, gamma)
+    want_v = oracle.anchor_similarity(v.float().cpu().numpy(), mode, gamma)
+    assert np.abs(out_k.cpu().numpy() - want_k).max() < SCORE_ATOL
+    assert np.abs(out_v.cpu().numpy() - want_v).max() < SCORE_ATOL
 
 
 def test_static_scratch_matches_workspace_path_twice_in_a_row():
