@@ -276,6 +276,13 @@ tf_status tf_set_scan_path(tf_ctx *ctx, int path);
  * default (about a second each).  For tests of the error path and for deployments that want a tighter bound. */
 tf_status tf_set_wait_limits(tf_ctx *ctx, int64_t max_polls, int64_t wait_cycles);
 
+/* Self-test of the bounded waits (the paper has no counterpart).  Launches one small CTA that waits, with the context's
+ * limits (capped at 1000 polls and 2e7 cycles), on an mbarrier nobody arrives at and on a record nobody writes, through the
+ * device functions the kernels wait with.  Afterwards tf_get_status returns TF_ERR_TIMEOUT (detail[1] = 901, 902 or 903:
+ * whichever wait gave up first), the context stays usable, and tf_clear_status resets it.  Harmless by construction: every
+ * one of these waits ends at its limit. */
+tf_status tf_wait_selftest(tf_ctx *ctx, void *stream);
+
 const char *tf_status_string(tf_status s);
 
 #ifdef __cplusplus

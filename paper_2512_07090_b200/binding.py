@@ -31,7 +31,7 @@ EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
            "tf_status_string", "tf_tail_policy", "tf_decode_step", "tf_set_scan_path", "tf_last_kernels",
-           "tf_set_wait_limits")
+           "tf_set_wait_limits", "tf_wait_selftest")
 
 
 class tf_shape(C.Structure):
@@ -255,6 +255,10 @@ class Context:
         """Limits of the kernels' bounded waits (negative: the default, about a second)."""
         _check(lib().tf_set_wait_limits(self._h, C.c_int64(int(max_polls)), C.c_int64(int(wait_cycles))),
                "tf_set_wait_limits")
+
+    def tf_wait_selftest(self):
+        """Make bounded waits run out on purpose (conditions nothing ever fulfils); tf_get_status then says TF_ERR_TIMEOUT."""
+        _check(lib().tf_wait_selftest(self._h, _stream()), "tf_wait_selftest")
 
     @property
     def launches(self) -> int:

@@ -81,6 +81,27 @@ __device__ __forceinline__ int first_kept_at_or_after(const int32_t* kept, int n
     return lo;
 }
 
+// ---- step a3: mean / population variance over heads, weight alpha (Eq. 2, either reading), fused score (Eq. 3) ----
+__device__ __forceinline__ float fuse_alpha(int mode, float var_k, float var_v, float eps) {
+    switch (mode) {
+        case TF_FUSE_EQ2_LITERAL: return (var_k + eps) / (var_k + var_v + 2.f * eps);
+        case TF_FUSE_KEY_ONLY: return 1.f;
+        case TF_FUSE_VALUE_ONLY: return 0.f;
+        case TF_FUSE_MEAN: return 0.5f;
+        default: return (var_v + eps) / (var_k + var_v + 2.f * eps);
+    }
+}
+__device__ __forceinline__ float fuse_score(int mode, float mean_k, float var_k, float mean_v, float var_v, float eps) {
+    const float alpha = fuse_alpha(mode, var_k, var_v, eps);
+    return (alpha * mean_k + (1.f - alpha) * mean_v) + 0.f;   // -0 -> +0
+}
+__device__ __forceinline__ void note_nan_score(DevStatus* st, float s, unsigned long long token) {
+    if (s != s && st) {
+        atomicAdd(&st->nan_count, 1ull);
+        report_error(st, TF_ERR_NAN_SCORE, token);
+    }
+}
+
 // ---- host-side launch bookkeeping --------------------------------------------------------------
 struct Strides3 { long long b, t, h; };
 

@@ -44,6 +44,55 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     return true;
 }
 
+// The same bounded wait for warps that may wait long next to warps that are busy: the hardware may park the thread for
+// up to the hinted time per try, and the clock and the abort flag are looked at once per 32 tries, so a waiting warp
+// costs few issue slots.
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                 long long budget_cycles, DevStatus* status, unsigned long long where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            uint32_t ok;
+            asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
+                         : "=r"(ok) : "r"(bar), "r"(parity), "r"(100000u) : "memory");
+            if (ok) return true;
+        }
+        if (*abort_flag) return false;
+        if (clock64() - t0 > budget_cycles) {
+            *abort_flag = 1;
+            report_error(status, TF_ERR_TIMEOUT, where);
+            return false;
+        }
+    }
+}
+
+// ---- 8-byte tagged packets {value, tag} in global memory: how one CTA hands a number to another --------------------
+__device__ __forceinline__ uint2 ld_packet2(const uint2* p) {
+    uint2 r;
+    asm volatile("ld.volatile.global.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
+    return r;
+}
+__device__ __forceinline__ void st_packet2(uint2* p, float v, unsigned int tag) {
+    asm volatile("st.volatile.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(__float_as_uint(v)), "r"(tag) : "memory");
+}
+__device__ __forceinline__ float wait_packet2(const uint2* p, uint2 first, unsigned int epoch, int max_polls,
+                                              DevStatus* status, unsigned long long where) {
+    uint2 r = first;
+    int polls = 0;
+    while (r.y != epoch) {
+        if (++polls > max_polls) {
+            report_error(status, TF_ERR_TIMEOUT, where);
+            r.x = 0u;
+            break;
+        }
+        __nanosleep(32);
+        r = ld_packet2(p);
+    }
+    return __uint_as_float(r.x);
+}
+
 // ---- TMA ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3) {

@@ -373,49 +373,44 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Step a3: one warp per token.  Mean and population variance over heads (two passes over the
-// registers), weight alpha per Eq. 2 (either reading), fused score per Eq. 3.
+// Step a3: G lanes per
+// token, G = 8, 16 or 32 by head count.  Mean and population variance over heads (two passes over the
+// similarities), weight alpha per Eq. 2 (either reading), fused score per Eq. 3.
 // ---------------------------------------------------------------------------------------------------
+template <int G>
 __global__ void __launch_bounds__(256) score_fuse_kernel(const float* __restrict__ sim_k,
                                                          const float* __restrict__ sim_v,
                                                          float* __restrict__ score, long long n_tokens,
                                                          int H, int mode, float eps, DevStatus* status) {
     grid_launch_dependents();   // a short kernel: the selection CTAs may become resident while it runs
     grid_dependency_wait();
-    const long long tok = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (tok >= n_tokens) return;
-    const float* ck = sim_k + tok * H;
-    const float* cv = sim_v + tok * H;
+    const long long tok = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const int lane = threadIdx.x & (G - 1);
+    const bool live = tok < n_tokens;               // whole groups are live or not; shuffles below stay inside a group
+    const float* ck = sim_k + (live ? tok : 0) * H;
+    const float* cv = sim_v + (live ? tok : 0) * H;
+    auto group_sum = [](float v) {
+#pragma unroll
+        for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        return v;
+    };
     float sk = 0.f, sv = 0.f;
-    for (int h = lane; h < H; h += 32) { sk += ck[h]; sv += cv[h]; }
+    for (int h = lane; h < H; h += G) { sk += ck[h]; sv += cv[h]; }
     const float inv = 1.f / (float)H;
-    sk = warp_sum(sk) * inv;
-    sv = warp_sum(sv) * inv;
+    sk = group_sum(sk) * inv;
+    sv = group_sum(sv) * inv;
     float vk = 0.f, vv = 0.f;
-    for (int h = lane; h < H; h += 32) {
+    for (int h = lane; h < H; h += G) {
         const float a = ck[h] - sk, b = cv[h] - sv;
         vk = fmaf(a, a, vk);
         vv = fmaf(b, b, vv);
     }
-    vk = warp_sum(vk) * inv;
-    vv = warp_sum(vv) * inv;
-    if (lane == 0) {
-        float alpha;
-        switch (mode) {
-            case TF_FUSE_EQ2_LITERAL: alpha = (vk + eps) / (vk + vv + 2.f * eps); break;
-            case TF_FUSE_KEY_ONLY: alpha = 1.f; break;
-            case TF_FUSE_VALUE_ONLY: alpha = 0.f; break;
-            case TF_FUSE_MEAN: alpha = 0.5f; break;
-            default: alpha = (vv + eps) / (vk + vv + 2.f * eps); break;
-        }
-        float s = alpha * sk + (1.f - alpha) * sv;
-        s += 0.f;   // -0 -> +0
+    vk = group_sum(vk) * inv;
+    vv = group_sum(vv) * inv;
+    if (lane == 0 && live) {
+        const float s = fuse_score(mode, sk, vk, sv, vv, eps);
         score[tok] = s;
-        if (s != s && status) {
-            atomicAdd(&status->nan_count, 1ull);
-            report_error(status, TF_ERR_NAN_SCORE, (unsigned long long)tok);
-        }
+        note_nan_score(status, s, (unsigned long long)tok);
     }
 }
 
@@ -424,9 +419,10 @@ cudaError_t launch_score_fuse(tf_ctx* ctx, const tf_shape& s, const tf_filter_pa
     const long long n = (long long)s.batch * s.seq;
     if (n == 0) return cudaSuccess;
     const float eps = p.var_eps > 0.f ? p.var_eps : 1e-8f;
-    const long long threads = n * 32;
-    const unsigned blocks = (unsigned)((threads + 255) / 256);
-    cudaError_t e = launch_dependent(score_fuse_kernel, dim3(blocks), dim3(256), 0, st, sim_k, sim_v, score, n,
+    const int G = s.n_kv_heads <= 8 ? 8 : (s.n_kv_heads <= 16 ? 16 : 32);
+    const unsigned blocks = (unsigned)((n * G + 255) / 256);
+    auto kernel = G == 8 ? score_fuse_kernel<8> : (G == 16 ? score_fuse_kernel<16> : score_fuse_kernel<32>);
+    cudaError_t e = launch_dependent(kernel, dim3(blocks), dim3(256), 0, st, sim_k, sim_v, score, n,
                                      s.n_kv_heads, p.fuse_mode, eps, ctx->dev_status);
     ctx->launches += 1;
     return e;

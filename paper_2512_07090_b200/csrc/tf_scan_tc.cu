@@ -13,6 +13,13 @@
 // cosines.  The fp32 instruction stream per (token, head) drops from ~130 to ~20 warp
 // instructions, which is what kept the plain kernel from reaching the memory roofline.
 //
+// EMA anchors (Eq. 1: anchor <- g anchor + (1-g) x, compared before it is updated) take the same products with
+// weights on the CUDA-core side.  With A0 the anchor before the tile:
+//   <x_i, A_i>    = g^i <x_i, A0> + (1-g) sum_{j<i} g^(i-1-j) G_ij     (row sums become Horner recurrences in g)
+//   ||A_{i+1}||^2 = g^2 ||A_i||^2 + 2 g (1-g) <x_i, A_i> + (1-g)^2 G_ii   (a prefix scan with ratio g^2)
+//   A_128         = g^128 A0 + (1-g) sum_j g^(127-j) x_j                 (the "ones" row of the small operand becomes
+//                                                                         three rows, 5-7, of bf16 terms of these weights)
+//
 // One CTA (128 threads) per (tile, tensor): K and V are independent here, and the smaller footprint
 // (32 KiB of rows, 64 TMEM columns, reused in turn for X^T 1, the two halves of G and X C) lets six CTAs
 // share an SM, so that the loads of some overlap the arithmetic of others.  Carries travel through tagged
@@ -43,34 +50,145 @@ __device__ __forceinline__ uint32_t bt_off(int n, int k) {
 }
 __device__ __forceinline__ unsigned short bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
 
+
+// ---- the two anchor forms: what differs between running sums and EMA anchors on the CUDA-core side ---------------
+// g^k for a small non-negative integer k (square-and-multiply: a few roundings, no transcendental)
+__device__ __forceinline__ float powi(float g, int k) {
+    float r = 1.f, b = g;
+    for (; k > 0; k >>= 1) {
+        if (k & 1) r *= b;
+        b *= b;
+    }
+    return r;
+}
+template <bool EMA> struct Anchor;
+template <> struct Anchor<false> {
+    __device__ __forceinline__ Anchor(float, int, int) {}
+    // thread i's row of G: a 32-column block wholly left of the diagonal / the block that holds the diagonal
+    __device__ __forceinline__ void full_block(const uint32_t* g, float& acc) const {
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int e = 0; e < 32; ++e) s4[e & 3] += __uint_as_float(g[e]);
+        acc += (s4[0] + s4[1]) + (s4[2] + s4[3]);
+    }
+    __device__ __forceinline__ void diag_block(const uint32_t* g, int lane, float& part, float& g_diag) const {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const float v = __uint_as_float(g[e]);
+            part += (e < lane) ? v : 0.f;
+            g_diag = (e == lane) ? v : g_diag;
+        }
+    }
+    __device__ __forceinline__ float dot(float u, float acc, float part) const { return u + (acc + part); }   // <x_i, P_i>
+    __device__ __forceinline__ float norm_step(float d, float g_diag) const { return fmaf(2.f, d, g_diag); } // ||P_{i+1}||^2 - ||P_i||^2
+    __device__ __forceinline__ float look_back(float A, float agg) const { return A + agg; }
+    __device__ __forceinline__ float carry_of(float prefix, float A, int) const { return prefix + A; }
+    __device__ __forceinline__ float sum_after(float carry, float agg, int) const { return carry + agg; }
+    __device__ __forceinline__ float agg_of(const uint32_t* r) const { return __uint_as_float(r[6]); }
+    // the block-wide exclusive prefix of the norm steps, seeded with n0; red: [4 warps] stride 2; sync: a barrier over the 128 threads
+    template <typename Sync>
+    __device__ __forceinline__ float norm_before(float b, float n0, int warp, int lane, volatile float* red, Sync sync) const {
+        float incl = b;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (lane == 31) red[warp * 2] = incl;
+        sync();
+        float off = n0;
+        for (int w2 = 0; w2 < warp; ++w2) off += red[w2 * 2];
+        return off + (incl - b);
+    }
+};
+template <> struct Anchor<true> {
+    float g, w, g8, g32, g128, pw_lane, pw_row, q32, q_lane, qs[5];
+    __device__ __forceinline__ Anchor(float gamma, int warp, int lane) {
+        g = gamma; w = 1.f - gamma;
+        g8 = powi(g, 8); g32 = powi(g, 32); g128 = powi(g, 128);
+        pw_lane = powi(g, lane); pw_row = powi(g, 32 * warp + lane);
+        q32 = powi(g, 64); q_lane = powi(g, 2 * lane);
+#pragma unroll
+        for (int k = 0; k < 5; ++k) qs[k] = powi(g, 2 << k);
+    }
+    // sum_e G[e] g^(31-e), then acc <- acc g^32 + that: after the blocks left of the diagonal, acc = sum_j g^(32 W - 1 - j) G_ij
+    __device__ __forceinline__ void full_block(const uint32_t* gr, float& acc) const {
+        float h[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            h[c] = __uint_as_float(gr[8 * c]);
+#pragma unroll
+            for (int e = 1; e < 8; ++e) h[c] = fmaf(h[c], g, __uint_as_float(gr[8 * c + e]));
+        }
+        const float r = fmaf(fmaf(fmaf(h[0], g8, h[1]), g8, h[2]), g8, h[3]);
+        acc = fmaf(acc, g32, r);
+    }
+    // sum_{e < lane} G[e] g^(lane-1-e)
+    __device__ __forceinline__ void diag_block(const uint32_t* gr, int lane, float& part, float& g_diag) const {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const float v = __uint_as_float(gr[e]);
+            part = (e < lane) ? fmaf(part, g, v) : part;
+            g_diag = (e == lane) ? v : g_diag;
+        }
+    }
+    __device__ __forceinline__ float dot(float u, float acc, float part) const { return fmaf(pw_row, u, w * fmaf(pw_lane, acc, part)); }
+    __device__ __forceinline__ float norm_step(float d, float g_diag) const { return fmaf(2.f * g * w, d, w * w * g_diag); }
+    __device__ __forceinline__ float look_back(float A, float agg) const { return fmaf(A, g128, agg); }
+    __device__ __forceinline__ float carry_of(float prefix, float A, int chunks) const {
+        float f = g128;
+        for (int m = 1; m < chunks; ++m) f *= g128;
+        return fmaf(f, prefix, A);
+    }
+    __device__ __forceinline__ float sum_after(float carry, float agg, int valid) const {
+        return fmaf(valid == kGT ? g128 : powi(g, valid), carry, agg);
+    }
+    __device__ __forceinline__ float agg_of(const uint32_t* r) const {
+        return (__uint_as_float(r[5]) + __uint_as_float(r[6])) + __uint_as_float(r[7]);
+    }
+    template <typename Sync>
+    __device__ __forceinline__ float norm_before(float b, float n0, int warp, int lane, volatile float* red, Sync sync) const {
+        float incl = b;                                  // sum_{j <= i, same warp} q^(i-j) b_j, q = g^2
+#pragma unroll
+        for (int k = 0; k < 5; ++k) {
+            const float n = __shfl_up_sync(0xffffffffu, incl, 1 << k);
+            if (lane >= (1 << k)) incl = fmaf(qs[k], n, incl);
+        }
+        if (lane == 31) red[warp * 2] = incl;
+        float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 0) excl = 0.f;
+        sync();
+        float cw = n0;                                   // ||A||^2 before this warp's first token
+        for (int w2 = 0; w2 < warp; ++w2) cw = fmaf(cw, q32, red[w2 * 2]);
+        return fmaf(q_lane, cw, excl);
+    }
+};
+// cosine of x_i to its anchor from d = <x_i, anchor sum>, xx = ||x_i||^2, pp = ||anchor sum||^2; the running-sum anchor
+// is the sum over cnt tokens divided by cnt (the division cancels unless a norm falls under its clamp), the EMA anchor is
+// the sum itself
+template <bool EMA>
+__device__ __forceinline__ float anchor_cosine(float d, float xx, float pp, long long cnt) {
+    if (cnt <= 0) return 0.f;
+    const float fc = EMA ? 1.f : (float)cnt, lim = kNormEps * kNormEps;
+    if (xx > lim && pp > lim * fc * fc) return d * rsqrtf(xx) * rsqrtf(pp);
+    const float sc = 1.f / fc;
+    return (d * sc) / (fmaxf(sqrtf(xx), kNormEps) * fmaxf(sqrtf(fmaxf(pp, 0.f)) * sc, kNormEps));
+}
+// the weight of token t of a tile with `valid` tokens in the tile's aggregate, as three bf16 terms
+template <bool EMA>
+__device__ __forceinline__ void agg_weight_terms(float gamma, int t, int valid, unsigned short out[3]) {
+    if (!EMA) { out[0] = 0x3f80; out[1] = 0; out[2] = 0; return; }      // 1, 0, 0
+    float wv = t < valid ? (1.f - gamma) * powi(gamma, valid - 1 - t) : 0.f;
+#pragma unroll
+    for (int n = 0; n < 3; ++n) {
+        out[n] = bf16_bits(wv);
+        wv -= __uint_as_float((uint32_t)out[n] << 16);
+    }
+}
+
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget_cycles,
                                          DevStatus* status, unsigned long long where) {
     return mbar_wait_bounded(bar, parity, abort_flag, budget_cycles, status, where);
-}
-
-// ---- 8-byte record packets {value, tag}: one tensor per CTA --------------------------------------------
-__device__ __forceinline__ uint2 ld_packet2(const uint2* p) {
-    uint2 r;
-    asm volatile("ld.volatile.global.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
-    return r;
-}
-__device__ __forceinline__ void st_packet2(uint2* p, float v, unsigned int tag) {
-    asm volatile("st.volatile.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(__float_as_uint(v)), "r"(tag) : "memory");
-}
-__device__ __forceinline__ float wait_packet2(const uint2* p, uint2 first, unsigned int epoch, int max_polls,
-                                              DevStatus* status, unsigned long long where) {
-    uint2 r = first;
-    int polls = 0;
-    while (r.y != epoch) {
-        if (++polls > max_polls) {
-            report_error(status, TF_ERR_TIMEOUT, where);
-            r.x = 0u;
-            break;
-        }
-        __nanosleep(32);
-        r = ld_packet2(p);
-    }
-    return __uint_as_float(r.x);
 }
 
 // One CTA per (tile, tensor): 32 KiB of rows, 64 TMEM columns, so six CTAs share an SM and their loads
@@ -83,6 +201,7 @@ constexpr uint32_t kIdescG64 = idesc(64, false);   // 64 columns of G at a time
 struct Gram1Params {
     int S, H, n_chains, n_chunks;
     int incl;
+    float gamma;                 // EMA anchors only
     const float* sum_in[2]; const long long* count_in;
     float* sum_out[2];
     float* sim[2];
@@ -95,6 +214,7 @@ struct Gram1Params {
     unsigned int n_work;         // (tile, tensor) pairs
 };
 
+template <bool EMA>
 __global__ void __launch_bounds__(128, 6)
 kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
     extern __shared__ uint8_t smem[];
@@ -125,7 +245,8 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     *reinterpret_cast<uint4*>(smem + kT1OffBt + tid * 32) = make_uint4(0, 0, 0, 0);
     *reinterpret_cast<uint4*>(smem + kT1OffBt + tid * 32 + 16) = make_uint4(0, 0, 0, 0);
     __syncthreads();
-    *reinterpret_cast<unsigned short*>(smem + kT1OffBt + bt_off(6, tid)) = 0x3f80;
+    if (!EMA) *reinterpret_cast<unsigned short*>(smem + kT1OffBt + bt_off(6, tid)) = 0x3f80;
+    const Anchor<EMA> an(p.gamma, warp, lane);
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kT1TmemCols);
     fence_proxy_async();
     tc_fence_before();
@@ -180,6 +301,15 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
             if (a0 + u < c) afirst[u] = ld_packet2(arec + u * astride);
     }
 
+    const int valid = min(kGT, p.S - c * kGT);       // tokens in this tile
+    if (EMA) {      // the aggregate's weights (rows 5-7 of the small operand, element = token) depend on the tile's length
+        unsigned short wt[3];
+        agg_weight_terms<EMA>(p.gamma, tid, valid, wt);
+#pragma unroll
+        for (int n = 0; n < 3; ++n) *reinterpret_cast<unsigned short*>(smem + kT1OffBt + bt_off(5 + n, tid)) = wt[n];
+        fence_proxy_async();
+        __syncthreads();
+    }
     uint32_t mma_phase = 0;
     wait_bar(bar_tma, 0, abort_flag, p.wait_cycles, p.status, 100);
 
@@ -200,7 +330,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
         tmem_ld8(tm_lane, r0);
         tmem_ld8(tm_lane + 16, r1);
         tmem_wait_ld();
-        agg = __uint_as_float(r0[6]) + __uint_as_float(r1[6]);
+        agg = an.agg_of(r0) + an.agg_of(r1);
     }
     if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, p.epoch);
     tc_fence_before();
@@ -216,18 +346,18 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
             float A = 0.f;
 #pragma unroll
             for (int u = 0; u < kGramAnchorEvery; ++u)       // requested while the tile was in flight
-                if (a0 + u < c) A += wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile);
-            carry = wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile) + A;
+                if (a0 + u < c) A = an.look_back(A, wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile));
+            carry = an.carry_of(wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile), A, c - a0);
         }
         if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
             st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, p.epoch);
-        if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = carry + agg;
+        if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = an.sum_after(carry, agg, valid);
     };
     const bool publishes_prefix = (c % kGramAnchorEvery == 0);
     if (publishes_prefix) resolve_carry();
 
     // ---- 2. G = X X^T, 64 columns at a time; thread i adds row i left of the diagonal ---------------------
-    float r_sum = 0.f, g_diag = 0.f;
+    float r_acc = 0.f, r_part = 0.f, g_diag = 0.f;
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
         if (tid == 0) {
@@ -248,19 +378,8 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
             uint32_t g[32];
             tmem_ld32(tm_lane + lc * 32, g);
             tmem_wait_ld();
-            if (cb < warp) {
-                float s4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int e = 0; e < 32; ++e) s4[e & 3] += __uint_as_float(g[e]);
-                r_sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float v = __uint_as_float(g[e]);
-                    r_sum += (e < lane) ? v : 0.f;
-                    g_diag = (e == lane) ? v : g_diag;
-                }
-            }
+            if (cb < warp) an.full_block(g, r_acc);
+            else an.diag_block(g, lane, r_part, g_diag);
         }
         tc_fence_before();
         __syncthreads();
@@ -300,38 +419,17 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
         tmem_ld8(tm_lane + 16, r1);
         tmem_wait_ld();
         auto f = [](uint32_t a, uint32_t b2) { return __uint_as_float(a) + __uint_as_float(b2); };
-        d = (f(r0[0], r1[0]) + f(r0[1], r1[1])) + f(r0[2], r1[2]) + r_sum;   // <x_i, P_i>
+        d = an.dot((f(r0[0], r1[0]) + f(r0[1], r1[1])) + f(r0[2], r1[2]), r_acc, r_part);   // <x_i, anchor before token i>
     }
 
-    // ---- 4. ||P_i||^2 by a block-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosine ----------
-    const float bi = fmaf(2.f, d, g_diag);
-    float incl_sum = bi;                           // inclusive warp scan
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float n = __shfl_up_sync(0xffffffffu, incl_sum, o);
-        if (lane >= o) incl_sum += n;
-    }
-    if (lane == 31) red[warp * 2 + 1] = incl_sum;
-    __syncthreads();
-    float off = c2;
-    for (int w2 = 0; w2 < warp; ++w2) off += red[w2 * 2 + 1];
-    float pp = off + (incl_sum - bi);              // ||P_i||^2 (exclusive)
+    // ---- 4. ||anchor||^2 before each token by a block-wide prefix scan of the norm steps, then the cosine ----------
+    const float bi = an.norm_step(d, g_diag);
+    float pp = an.norm_before(bi, c2, warp, lane, red + 1, [] { __syncthreads(); });
     const int t_tok = c * kGT + tid;
     if (t_tok < p.S) {
         if (p.incl) { d += g_diag; pp += bi; }
         const long long cnt = (p.count_in ? p.count_in[b] : 0ll) + t_tok + (p.incl ? 1 : 0);
-        float cosv = 0.f;
-        if (cnt > 0) {
-            // anchor = sum / cnt; the 1 / cnt cancels unless a norm falls under its clamp
-            const float fc = (float)cnt, lim = kNormEps * kNormEps;
-            if (g_diag > lim && pp > lim * fc * fc) {
-                cosv = d * rsqrtf(g_diag) * rsqrtf(pp);
-            } else {
-                const float s = 1.f / fc;
-                cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pp, 0.f)) * s, kNormEps));
-            }
-        }
-        p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = cosv;
+        p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = anchor_cosine<EMA>(d, g_diag, pp, cnt);
     }
 
     tc_fence_before();
@@ -392,27 +490,9 @@ __device__ __forceinline__ void mma_burst(std::integer_sequence<int, KK...>, uin
                                           uint32_t b_lo, uint32_t b_hi, uint32_t id) {
     (mma_step<(A_MN ? (uint32_t)(KK * 16 * 128 >> 4) : kmaj_step(KK, BLOCK)), kmaj_step(KK, BLOCK), (KK > 0)>(d_tmem, a_lo, a_hi, b_lo, b_hi, id), ...);
 }
-// mbarrier wait for the persistent kernel: the hardware may park the thread for up to the hinted time per try, and
-// the clock and the abort flag are looked at once per 32 tries, so a waiting warp costs few issue slots
 __device__ __forceinline__ bool wait_bar_parked(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget_cycles,
                                                 DevStatus* status, unsigned long long where) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 32; ++i) {
-            uint32_t ok;
-            asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
-                         : "=r"(ok) : "r"(bar), "r"(parity), "r"(100000u) : "memory");
-            if (ok) return true;
-        }
-        if (*abort_flag) return false;
-        if (clock64() - t0 > budget_cycles) {
-            *abort_flag = 1;
-            report_error(status, TF_ERR_TIMEOUT, where);
-            return false;
-        }
-    }
+    return mbar_wait_parked(bar, parity, abort_flag, budget_cycles, status, where);
 }
 __device__ __forceinline__ void worker_sync(int w) { asm volatile("bar.sync %0, 128;" :: "r"(w + 1) : "memory"); }
 // byte offset, from the worker's base, of element (row n, index k) of the small operand
@@ -420,6 +500,7 @@ __device__ __forceinline__ uint32_t pbt_off(int n, int k) {
     return (uint32_t)((k >> 6) * kPBlock + kHalf + n * 128 + ((((k & 63) >> 3) ^ (n & 7)) << 4) + (k & 7) * 2);
 }
 
+template <bool EMA>
 __global__ void __launch_bounds__(kPThreads, 1)
 kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CUtensorMap mapK,
                                 const __grid_constant__ CUtensorMap mapV) {
@@ -458,7 +539,19 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         *reinterpret_cast<uint4*>(dst + 16) = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
-    *reinterpret_cast<unsigned short*>(my + pbt_off(6, tid)) = 0x3f80;
+    const Anchor<EMA> an(p.gamma, warp, lane);
+    int w_valid = kGT;                // the tile length the aggregate's weights (rows 5-7, element = token) are written for
+    auto write_agg_weights = [&](int valid) {
+        unsigned short wt[3];
+        agg_weight_terms<EMA>(p.gamma, tid, valid, wt);
+        if (EMA) {
+#pragma unroll
+            for (int n = 0; n < 3; ++n) *reinterpret_cast<unsigned short*>(my + pbt_off(5 + n, tid)) = wt[n];
+        } else {
+            *reinterpret_cast<unsigned short*>(my + pbt_off(6, tid)) = wt[0];
+        }
+    };
+    write_agg_weights(kGT);
     if (threadIdx.x < 32) tmem_alloc(smem_u32(tmem_slot), kPTmemCols);
     fence_proxy_async();
     tc_fence_before();
@@ -509,6 +602,13 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         unsigned int t_next = kPNoTile;
         if (tid == 0) t_next = draw();                       // the answer is needed only when this tile's products are done
         const long long cnt0 = p.count_in ? p.count_in[b] : 0ll;
+        const int valid = min(kGT, p.S - c * kGT);           // tokens in this tile
+        if (EMA && valid != w_valid) {   // a shorter (last) tile, or the first full one after it: other weights in the aggregate
+            write_agg_weights(valid);
+            w_valid = valid;
+            fence_proxy_async();
+            worker_sync(w);
+        }
 
         wait_bar_parked(bar_tma, tile_phase, abort_flag, p.wait_cycles, p.status, 200);
 
@@ -541,7 +641,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             uint32_t r0[8];
             tmem_ld8(tm_s + lane_off, r0);
             tmem_wait_ld();
-            agg = __uint_as_float(r0[6]);
+            agg = an.agg_of(r0);
         }
         if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, p.epoch);
 
@@ -553,12 +653,12 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             float A = 0.f;
 #pragma unroll
             for (int u = 0; u <= kPLookBack; ++u)
-                if (a0 + u < c) A += wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile);
-            carry = wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile) + A;
+                if (a0 + u < c) A = an.look_back(A, wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile));
+            carry = an.carry_of(wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile), A, c - a0);
         }
         if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
             st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, p.epoch);
-        if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = carry + agg;
+        if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = an.sum_after(carry, agg, valid);
         {   // the carry as c1 + c2 + c3 (bf16 each) into rows 0-2 of the small operand
             float cr = carry;
 #pragma unroll
@@ -572,7 +672,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
         if (lane == 0) red[warp * 2] = c2;
 
         // thread i adds row i of a 64-column half of G left of the diagonal
-        float r_sum = 0.f, g_diag = 0.f;
+        float r_acc = 0.f, r_part = 0.f, g_diag = 0.f;
         auto add_half = [&](int hh) {
 #pragma unroll
             for (int lc = 0; lc < 2; ++lc) {
@@ -581,19 +681,8 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
                 uint32_t g[32];
                 tmem_ld32(tm_g + lane_off + lc * 32, g);
                 tmem_wait_ld();
-                if (cb < warp) {
-                    float s4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) s4[e & 3] += __uint_as_float(g[e]);
-                    r_sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const float v = __uint_as_float(g[e]);
-                        r_sum += (e < lane) ? v : 0.f;
-                        g_diag = (e == lane) ? v : g_diag;
-                    }
-                }
+                if (cb < warp) an.full_block(g, r_acc);
+                else an.diag_block(g, lane, r_part, g_diag);
             }
         };
         wait_bar_parked(bar_g, 0, abort_flag, p.wait_cycles, p.status, 202);
@@ -619,39 +708,18 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             uint32_t r0[8];
             tmem_ld8(tm_s + lane_off, r0);
             tmem_wait_ld();
-            d = (__uint_as_float(r0[0]) + __uint_as_float(r0[1])) + __uint_as_float(r0[2]) + r_sum;   // <x_i, P_i>
+            d = an.dot((__uint_as_float(r0[0]) + __uint_as_float(r0[1])) + __uint_as_float(r0[2]), r_acc, r_part);   // <x_i, anchor before token i>
         }
 
-        // ---- ||P_i||^2 by a worker-wide exclusive prefix sum of 2 <x_i,P_i> + G_ii, then the cosine -------------
-        const float bi = fmaf(2.f, d, g_diag);
-        float incl_sum = bi;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float n = __shfl_up_sync(0xffffffffu, incl_sum, o);
-            if (lane >= o) incl_sum += n;
-        }
-        if (lane == 31) red[warp * 2 + 1] = incl_sum;
+        // ---- ||anchor||^2 before each token by a worker-wide prefix scan of the norm steps, then the cosine -------------
+        const float bi = an.norm_step(d, g_diag);
         tc_fence_before();
-        worker_sync(w);
-        float off = c2;
-        for (int w2 = 0; w2 < warp; ++w2) off += red[w2 * 2 + 1];
-        float pn = off + (incl_sum - bi);              // ||P_i||^2 (exclusive)
+        float pn = an.norm_before(bi, c2, warp, lane, red + 1, [w] { worker_sync(w); });
         const int t_tok = c * kGT + tid;
         if (t_tok < p.S) {
             if (p.incl) { d += g_diag; pn += bi; }
             const long long cnt = cnt0 + t_tok + (p.incl ? 1 : 0);
-            float cosv = 0.f;
-            if (cnt > 0) {
-                // anchor = sum / cnt; the 1 / cnt cancels unless a norm falls under its clamp
-                const float fc = (float)cnt, lim = kNormEps * kNormEps;
-                if (g_diag > lim && pn > lim * fc * fc) {
-                    cosv = d * rsqrtf(g_diag) * rsqrtf(pn);
-                } else {
-                    const float s = 1.f / fc;
-                    cosv = (d * s) / (fmaxf(sqrtf(g_diag), kNormEps) * fmaxf(sqrtf(fmaxf(pn, 0.f)) * s, kNormEps));
-                }
-            }
-            p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = cosv;
+            p.sim[x][((size_t)b * p.S + t_tok) * p.H + h] = anchor_cosine<EMA>(d, g_diag, pn, cnt);
         }
         cur = make_uint4(s_next[0], s_next[1], s_next[2], s_next[3]);   // rewritten, like red[], only after the next tile's first worker barrier
     }
@@ -670,7 +738,8 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
 }  // namespace
 
 bool kv_stats_gram_usable(const tf_shape& s, const tf_filter_params& p) {
-    return s.dtype == TF_BF16 && p.anchor_mode != TF_ANCHOR_EMA;
+    (void)p;
+    return s.dtype == TF_BF16;      // every anchor mode: running sums (past / inclusive mean) and EMA
 }
 
 namespace {
@@ -721,13 +790,16 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     static bool attr_set_dev[kDeviceFlagSlots] = {};      // function attributes are per device
     bool& attr_set = attr_set_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kv_stats_gram1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kT1Smem);
+        cudaError_t e = cudaFuncSetAttribute(kv_stats_gram1_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kT1Smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kv_stats_gram1_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kT1Smem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     Gram1Params gp{};
     gp.S = s.seq; gp.H = s.n_kv_heads; gp.n_chains = gl.n_chains; gp.n_chunks = gl.n_chunks;
     gp.incl = (p.anchor_mode == TF_ANCHOR_INCL_MEAN);
+    const bool ema = (p.anchor_mode == TF_ANCHOR_EMA);
+    gp.gamma = ema ? p.gamma : 1.f;
     if (carry) {
         gp.sum_in[0] = carry->sum_k_in; gp.sum_in[1] = carry->sum_v_in;
         gp.count_in = reinterpret_cast<const long long*>(carry->count_in);
@@ -756,17 +828,20 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
         static bool attr_set_p_dev[kDeviceFlagSlots] = {};
         bool& attr_set_p = attr_set_p_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
         if (!attr_set_p) {
-            e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
+            e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(kv_stats_gram_persistent_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem);
             if (e != cudaSuccess) return e;
             attr_set_p = true;
         }
         const unsigned int grid = std::min<unsigned int>((unsigned int)sms, (gp.n_work + kPWorkers - 1) / kPWorkers);
         GramPParams pp{};
         pp.g = gp;
-        e = launch_dependent(kv_stats_gram_persistent_kernel, dim3(grid), dim3(kPThreads), kPSmem, st, pp, mk, mv);
+        e = ema ? launch_dependent(kv_stats_gram_persistent_kernel<true>, dim3(grid), dim3(kPThreads), kPSmem, st, pp, mk, mv)
+                : launch_dependent(kv_stats_gram_persistent_kernel<false>, dim3(grid), dim3(kPThreads), kPSmem, st, pp, mk, mv);
         ctx->last_scan_kernel = TF_KERNEL_SCAN_GRAM_PERSISTENT;
     } else {
-        e = launch_dependent(kv_stats_gram1_kernel, dim3(gp.n_work), dim3(128), kT1Smem, st, gp, mk, mv);
+        e = ema ? launch_dependent(kv_stats_gram1_kernel<true>, dim3(gp.n_work), dim3(128), kT1Smem, st, gp, mk, mv)
+                : launch_dependent(kv_stats_gram1_kernel<false>, dim3(gp.n_work), dim3(128), kT1Smem, st, gp, mk, mv);
         ctx->last_scan_kernel = TF_KERNEL_SCAN_GRAM_TILE;
     }
     ctx->launches += 1;

@@ -8,7 +8,8 @@
 // The retained positions are compacted in ascending order with warp ballots and a block-wide
 // prefix sum.  For sequences of up to 16384 tokens every thread keeps its scores in registers
 // (token i*1024 + tid in slot i), so the passes run out of registers and shared memory; longer
-// sequences re-read the scores from global memory on each pass.  (Producing the scores inside this
+// sequences stage the scores in shared memory (up to 51200 tokens) or re-read them from global memory
+// on each pass.  (Producing the scores inside this
 // kernel as well was measured: one CTA per sequence reads the per-head similarities far too slowly.)
 #include <math_constants.h>
 
@@ -36,6 +37,7 @@ struct SelectParams {
     const float* threshold;    // [B] (threshold mode)
     int S, warmup, mode;
     long long p_target;        // floor(ratio*S), computed on the host in double
+    int stage;                 // re-reading form only: 1 = the launch has S floats of dynamic shared memory for the scores
     uint8_t* keep_mask; int32_t* kept_idx; int32_t* n_kept; float* theta;
 };
 
@@ -72,6 +74,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     grid_dependency_wait();
     const int b = blockIdx.x, tid = threadIdx.x, S = p.S;
     const float* sc = p.score + (size_t)b * S;
+    if (KPT == 0 && p.stage) {   // too many scores for registers: the passes below read them from shared memory
+        extern __shared__ float s_scores[];
+        for (int t = tid; t < S; t += kSelThreads) s_scores[t] = sc[t];
+        __syncthreads();
+        sc = s_scores;
+    }
     const uint8_t* el = p.eligible ? p.eligible + (size_t)b * S : nullptr;
     constexpr int NR = KPT > 0 ? KPT : 1;
     float sreg[NR];
@@ -352,7 +360,23 @@ cudaError_t launch_select_form(const SelectParams& sp, int batch, cudaStream_t s
     if (S <= 4 * kSelThreads) return launch_dependent(select_kernel<4>, grid, block, 0, st, sp);
     if (S <= 8 * kSelThreads) return launch_dependent(select_kernel<8>, grid, block, 0, st, sp);
     if (S <= 16 * kSelThreads) return launch_dependent(select_kernel<16>, grid, block, 0, st, sp);
-    return launch_dependent(select_kernel<0>, grid, block, 0, st, sp);
+    // longer sequences: the scores go to shared memory once (up to 200 KiB = 51200 tokens), else every pass re-reads them
+    constexpr size_t kStageMax = 200 << 10;
+    SelectParams sp2 = sp;
+    const size_t need = (size_t)S * sizeof(float);
+    sp2.stage = need <= kStageMax ? 1 : 0;
+    if (sp2.stage) {
+        static bool attr_set_dev[kDeviceFlagSlots] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        bool& attr_set = attr_set_dev[dev >= 0 && dev < kDeviceFlagSlots ? dev : 0];
+        if (!attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(select_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStageMax);
+            if (e != cudaSuccess) return e;
+            attr_set = true;
+        }
+    }
+    return launch_dependent(select_kernel<0>, grid, block, sp2.stage ? need : 0, st, sp2);
 }
 }  // namespace
 
