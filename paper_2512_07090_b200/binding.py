@@ -25,7 +25,7 @@ TF_SELECT_RATIO, TF_SELECT_THRESHOLD = 0, 1
 TF_KV_ALL, TF_KV_RETAINED = 0, 1
 TF_STATIC_SCRATCH_BYTES = 8 << 20
 (TF_KERNEL_NONE, TF_KERNEL_SCAN_PLAIN, TF_KERNEL_SCAN_GRAM_TILE, TF_KERNEL_SCAN_GRAM_PERSISTENT) = range(4)
-TF_KERNEL_ATTN_SIMT, TF_KERNEL_ATTN_TC_SHARED, TF_KERNEL_ATTN_TC_SPLIT = 10, 11, 12
+TF_KERNEL_ATTN_SIMT, TF_KERNEL_ATTN_TC_SHARED, TF_KERNEL_ATTN_TC_SPLIT, TF_KERNEL_ATTN_TC_SINGLE = 10, 11, 12, 13
 
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
@@ -238,7 +238,8 @@ class Context:
         _check(lib().tf_clear_status(self._h), "tf_clear_status")
 
     def tf_set_attention_path(self, path):
-        """0 / False: CUDA-core kernel; 1 / True: tensor-core kernel (form chosen by size); 2: shared form; 3: split form."""
+        """0 / False: CUDA-core kernel; 1 / True: tensor-core kernel (form chosen by size); 2: shared form; 3: split form;
+        4: single form (one Q tile and one softmax group per CTA, two CTAs per SM)."""
         _check(lib().tf_set_attention_path(self._h, C.c_int(int(path))), "tf_set_attention_path")
 
     def tf_set_scan_path(self, path: int):

@@ -126,6 +126,78 @@ __device__ __forceinline__ uint32_t swz(int r, int cc) {
 }
 
 
+// One thread's share (a row of 128 scores) of one K/V tile of 128 keys starting at key j0: S from TMEM, masking by the
+// row's own visible range lo .. hi, running reference maximum, exponentials, P as bf16 pairs back into TMEM over the first
+// 64 columns of S, running sum.  O (when it exists already) is rescaled when the reference maximum moves.
+__device__ __forceinline__ void softmax_tile(uint32_t tm_s, uint32_t tm_o, int lo, int hi, int j0, float scale_log2,
+                                             bool have_o, float& m_ref, float& l_run) {
+    uint32_t sreg[128];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, sreg + c * 32);
+    tmem_wait_ld();
+    const bool full = (j0 >= lo) && (j0 + kTileN - 1 <= hi);
+    if (!full) {   // columns below c_lo or above c_hi are invisible to this row: -inf
+        const int c_lo = lo - j0, c_hi = hi - j0;
+        if (c_lo <= 0) {
+#pragma unroll
+            for (int c = 0; c < 128; ++c) if (c > c_hi) sreg[c] = 0xff800000u;
+        } else if (c_hi >= kTileN - 1) {
+#pragma unroll
+            for (int c = 0; c < 128; ++c) if (c < c_lo) sreg[c] = 0xff800000u;
+        } else {
+#pragma unroll
+            for (int c = 0; c < 128; ++c) if (c < c_lo || c > c_hi) sreg[c] = 0xff800000u;
+        }
+    }
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains, not one of 128
+#pragma unroll
+    for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            mx4[u] = max3(mx4[u], __uint_as_float(sreg[c + 2 * u]), __uint_as_float(sreg[c + 2 * u + 1]));
+    }
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+    __syncwarp();   // rows take different masking branches; the TMEM accesses below are warp-wide
+    // move the reference maximum only when the tile maximum exceeds it by 2^8 or more
+    const float m_tile = mx * scale_log2;
+    const bool move = m_tile > m_ref + kRescaleThreshold;   // also true on the first visible key (m_ref = -inf)
+    const float m_new = move ? m_tile : m_ref;
+    const float corr = move ? ex2(m_ref - m_new) : 1.f;
+    if (have_o && __any_sync(0xffffffffu, move)) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tm_o + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * corr);
+            tmem_st32(tm_o + c * 32, o);
+        }
+    }
+    m_ref = m_new;
+    const float m_safe = (m_ref == -INFINITY) ? 0.f : m_ref;
+    const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m_safe, -m_safe);
+    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(sreg[h * 64 + 2 * c]), __uint_as_float(sreg[h * 64 + 2 * c + 1])), sc2, nm2), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            acc[c & 3] = add2(acc[c & 3], pack2(p0, p1));
+            pk[c] = pack_bf16(p0, p1);
+        }
+        tmem_st32(tm_s + h * 32, pk);   // P_i over the first 64 columns of S_i
+    }
+    float a0, a1, a2, a3;
+    unpack2(add2(acc[0], acc[1]), a0, a1);
+    unpack2(add2(acc[2], acc[3]), a2, a3);
+    const float psum = (a0 + a1) + (a2 + a3);
+    l_run = fmaf(l_run, corr, psum);
+}
+
 template <bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
@@ -379,71 +451,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             mbar_wait(bar_s + 8 * i, c_it & 1, abort_flag, p.wait_cycles, p.status, 30 + i);
             __syncwarp();
             tc_fence_after();
-            uint32_t sreg[128];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tm_s + c * 32, sreg + c * 32);
-            tmem_wait_ld();
-            const bool full = (j0 >= lo) && (j0 + kTileN - 1 <= hi);
-            if (!full) {   // columns below c_lo or above c_hi are invisible to this row: -inf
-                const int c_lo = lo - j0, c_hi = hi - j0;
-                if (c_lo <= 0) {
-#pragma unroll
-                    for (int c = 0; c < 128; ++c) if (c > c_hi) sreg[c] = 0xff800000u;
-                } else if (c_hi >= kTileN - 1) {
-#pragma unroll
-                    for (int c = 0; c < 128; ++c) if (c < c_lo) sreg[c] = 0xff800000u;
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 128; ++c) if (c < c_lo || c > c_hi) sreg[c] = 0xff800000u;
-                }
-            }
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains, not one of 128
-#pragma unroll
-            for (int c = 0; c < 128; c += 8) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    mx4[u] = max3(mx4[u], __uint_as_float(sreg[c + 2 * u]), __uint_as_float(sreg[c + 2 * u + 1]));
-            }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            __syncwarp();   // rows take different masking branches; the TMEM accesses below are warp-wide
-            // move the reference maximum only when the tile maximum exceeds it by 2^8 or more
-            const float m_tile = mx * p.scale_log2;
-            const bool move = m_tile > m_ref + kRescaleThreshold;   // also true on the first visible key (m_ref = -inf)
-            const float m_new = move ? m_tile : m_ref;
-            const float corr = move ? ex2(m_ref - m_new) : 1.f;
-            if (c_it > 0 && __any_sync(0xffffffffu, move)) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tm_o + c * 32, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * corr);
-                    tmem_st32(tm_o + c * 32, o);
-                }
-            }
-            m_ref = m_new;
-            const float m_safe = (m_ref == -INFINITY) ? 0.f : m_ref;
-            const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_safe, -m_safe);
-            uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t pk[32];
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    float x0, x1;
-                    unpack2(fma2(pack2(__uint_as_float(sreg[h * 64 + 2 * c]), __uint_as_float(sreg[h * 64 + 2 * c + 1])), sc2, nm2), x0, x1);
-                    const float p0 = ex2(x0), p1 = ex2(x1);
-                    acc[c & 3] = add2(acc[c & 3], pack2(p0, p1));
-                    pk[c] = pack_bf16(p0, p1);
-                }
-                tmem_st32(tm_s + h * 32, pk);   // P_i over the first 64 columns of S_i
-            }
-            float a0, a1, a2, a3;
-            unpack2(add2(acc[0], acc[1]), a0, a1);
-            unpack2(add2(acc[2], acc[3]), a2, a3);
-            const float psum = (a0 + a1) + (a2 + a3);
-            l_run = fmaf(l_run, corr, psum);
+            softmax_tile(tm_s, tm_o, lo, hi, j0, p.scale_log2, c_it > 0, m_ref, l_run);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p + 8 * i);
@@ -549,6 +557,250 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Single form: ONE 128-row Q tile and ONE softmax group per CTA -- 256 threads, 256 TMEM columns (S | O) and 96 KiB
+// of shared memory (the Q tile, one K slot, one V slot), so that TWO CTAs share an SM.  What the two softmax groups
+// of the other forms do for each other inside a CTA (one exponentiates while the tensor pipe works for the other),
+// two independent CTAs do here, and in addition the set-up, Q gather and epilogue of one CTA run under the steady
+// state of its neighbour: the fixed cost per CTA, a third of all SM time on small problems, is no longer idle time.
+// Every Q tile streams its own K/V tiles (as in the split form), so this form suits problems whose K/V traffic the
+// L2 can feed twice over.  Warp roles: warps 0-3 softmax (thread r owns row r), warp 4 issues the products, warp 5
+// the TMA loads, warps 6-7 zero the output rows of pruned tokens.
+//   K(j+1) is requested as soon as Q K_j^T has read K(j), V(j+1) as soon as P V_j has read V(j): with one slot each
+//   the loads run under the softmax of tile j and the products of the neighbouring CTA.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kThreads1 = 256;
+constexpr int kMmaWarp1 = 4, kTmaWarp1 = 5;
+constexpr uint32_t kTmemCols1 = 256;
+constexpr int kOffQ1 = 0, kOffK1 = kTileBytes, kOffV1 = 2 * kTileBytes, kOffBar1 = 3 * kTileBytes;
+constexpr int kSmemBytes1 = kOffBar1 + 256;      // the dynamic segment must start 1024-byte aligned (checked)
+constexpr int kRegs1 = 128;                      // registers per thread at launch: 256 x 128 = 128 x 200 + 128 x 56
+
+__global__ void __launch_bounds__(kThreads1, 2)
+attention_tc_single_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
+    extern __shared__ uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {   // the swizzled operand layout needs it; nothing has been started yet
+        if (tid == 0) report_error(p.status, TF_ERR_TIMEOUT, 399);
+        return;
+    }
+    const uint32_t bar_q = sbase + kOffBar1;              // Q tile written
+    const uint32_t bar_fk = bar_q + 8, bar_fv = bar_q + 16;   // K / V slot filled by TMA
+    const uint32_t bar_ek = bar_q + 24, bar_ev = bar_q + 32;  // K / V slot consumed by the products
+    const uint32_t bar_s = bar_q + 40, bar_p = bar_q + 48, bar_o = bar_q + 56;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar1 + 64);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar1 + 72);
+    if (tid == 0) {
+        mbar_init(bar_q, kTileM);
+        mbar_init(bar_fk, 1); mbar_init(bar_fv, 1); mbar_init(bar_ek, 1); mbar_init(bar_ev, 1);
+        mbar_init(bar_s, 1); mbar_init(bar_p, kTileM); mbar_init(bar_o, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncwarp();
+    if (warp == kMmaWarp1) tmem_alloc(smem_u32(tmem_slot), kTmemCols1);
+    grid_dependency_wait();   // kept_idx / n_kept come from the kernel before this one
+    const int n_bh = (int)(gridDim.x / (unsigned)p.n_row_blocks);
+    const int rb = p.heads_fastest ? (int)blockIdx.x / n_bh : (int)blockIdx.x % p.n_row_blocks;
+    const int bh = p.heads_fastest ? (int)blockIdx.x % n_bh : (int)blockIdx.x / p.n_row_blocks;
+    int blk = p.first_pair - rb;          // heaviest expected row block first, blocks expected to be empty last
+    if (blk < 0) blk += p.n_row_blocks;
+    const int qh = bh % p.Hq, b = bh / p.Hq;
+    const int nk = p.n_kept[b];
+    const int slot0 = blk * kTileM;
+    const int32_t* kept = p.kept_idx + (size_t)b * p.S;
+    __nv_bfloat16* Ob = p.O + (long long)b * p.os.b + (long long)qh * p.os.h;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    if (slot0 >= max(nk, 1) || nk == 0) {   // no retained row in this block (CTA-uniform)
+        if (slot0 < max(nk, 1)) {           // nothing retained at all: the whole head is zero
+            for (int i = tid; i < p.S * 16; i += kThreads1)
+                *reinterpret_cast<uint4*>(Ob + (long long)(i >> 4) * p.os.t + (i & 15) * 8) = zero4;
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        if (warp == kMmaWarp1) tmem_dealloc(*tmem_slot, kTmemCols1);
+        return;
+    }
+    // retained indices of the Q rows this thread gathers (16 lanes per 256-byte row, the 4 softmax warps take 8 rows per
+    // round) and of its own row
+    constexpr int kRounds = kTileM / 8;
+    int tq[kRounds];
+    int t_row = -1;
+    if (warp < kMmaWarp1) {
+#pragma unroll
+        for (int it = 0; it < kRounds; ++it) {
+            const int s_q = slot0 + it * 8 + warp * 2 + (lane >> 4);
+            tq[it] = s_q < nk ? kept[s_q] : -1;
+        }
+        if (slot0 + tid < nk) t_row = kept[slot0 + tid];
+    }
+    // which K/V tiles the Q tile needs (CTA-uniform): J0 .. J1 - 1
+    int J0, J1;
+    {
+        const int s_last = min(slot0 + kTileM, nk) - 1;
+        const int t_first = kept[slot0], t_last = kept[s_last];
+        int k_first = p.window > 0 ? max(0, t_first - p.window + 1) : 0;
+        int k_last = t_last;
+        if (p.compact) {   // keys are entries of the retained list
+            k_first = p.window > 0 ? first_kept_at_or_after(kept, slot0 + 1, k_first) : 0;
+            k_last = s_last;
+        }
+        J0 = k_first / kTileN;
+        J1 = k_last / kTileN + 1;
+    }
+    const int kh = qh / (p.Hq / p.Hkv);
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp >= kMmaWarp1) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        if (warp > kTmaWarp1) {
+            // ================================ zero fill ====================================================
+            const int g4 = (tid - (kTmaWarp1 + 1) * 32) >> 4, l16 = tid & 15;
+            const int s_end = min(slot0 + kTileM, nk);
+            for (int s_z = slot0 + g4; s_z < s_end; s_z += 4) {
+                const int prev = s_z == 0 ? -1 : kept[s_z - 1], cur = kept[s_z];
+                for (int t = prev + 1; t < cur; ++t) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + l16 * 8) = zero4;
+                if (s_z == nk - 1)
+                    for (int t = cur + 1; t < p.S; ++t) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + l16 * 8) = zero4;
+            }
+        } else if (warp == kTmaWarp1) {
+            // ================================ TMA producer ================================================
+            if (lane == 0) {
+                for (int j = J0; j < J1; ++j) {
+                    const int n = j - J0;
+                    if (n > 0) mbar_wait(bar_ek, (n - 1) & 1, abort_flag, p.wait_cycles, p.status, 10);
+                    mbar_expect_tx(bar_fk, kTileBytes);
+                    tma_load_4d(sbase + kOffK1, &mapK, bar_fk, 0, kh, j * kTileN, b);
+                    tma_load_4d(sbase + kOffK1 + kHalfBytes, &mapK, bar_fk, 64, kh, j * kTileN, b);
+                    if (n > 0) mbar_wait(bar_ev, (n - 1) & 1, abort_flag, p.wait_cycles, p.status, 11);
+                    mbar_expect_tx(bar_fv, kTileBytes);
+                    tma_load_4d(sbase + kOffV1, &mapV, bar_fv, 0, kh, j * kTileN, b);
+                    tma_load_4d(sbase + kOffV1 + kHalfBytes, &mapV, bar_fv, 64, kh, j * kTileN, b);
+                }
+            }
+        } else {
+            // ================================ MMA issuer ==================================================
+            if (lane == 0) {
+                auto issue_qk = [&]() {           // S = Q K_j^T : 8 steps of 16 dims
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                        mma_ss(tmem, desc_kmajor(sbase + kOffQ1 + off), desc_kmajor(sbase + kOffK1 + off), kIdescQK, kk > 0);
+                    }
+                    mma_commit(bar_s);
+                    mma_commit(bar_ek);
+                };
+                mbar_wait(bar_q, 0, abort_flag, p.wait_cycles, p.status, 20);
+                mbar_wait(bar_fk, 0, abort_flag, p.wait_cycles, p.status, 21);
+                tc_fence_after();
+                issue_qk();
+                for (int j = J0; j < J1; ++j) {
+                    const int n = j - J0;
+                    mbar_wait(bar_fv, n & 1, abort_flag, p.wait_cycles, p.status, 22);
+                    mbar_wait(bar_p, n & 1, abort_flag, p.wait_cycles, p.status, 24);
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)    // O (+)= P V_j : 8 steps of 16 keys
+                        mma_ts(tmem + 128, tmem + kk * 8, desc_mnmajor(sbase + kOffV1 + kk * 16 * 128, kHalfBytes), kIdescPV,
+                               (n > 0 || kk > 0) ? 1u : 0u);
+                    mma_commit(bar_ev);
+                    if (j + 1 < J1) {
+                        mbar_wait(bar_fk, (n + 1) & 1, abort_flag, p.wait_cycles, p.status, 23);
+                        tc_fence_after();
+                        issue_qk();
+                    }
+                }
+                mma_commit(bar_o);
+            }
+        }
+    } else {
+        // ================================ softmax group ================================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+        const int r = tid;                        // row within the tile
+        const int slot = slot0 + r;
+        const bool valid = slot < nk;
+        int hi = t_row;                                                           // visible keys: lo .. hi
+        int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
+        if (p.compact && valid) {
+            lo = p.window > 0 ? first_kept_at_or_after(kept, slot + 1, lo) : 0;
+            hi = slot;
+        }
+        {   // gather the Q rows into the swizzled K-major operand layout
+            const int sub = lane >> 4, cc = lane & 15;
+            uint4 qv[kRounds];
+            const __nv_bfloat16* qbase = p.Q + (long long)b * p.qs.b + (long long)qh * p.qs.h + cc * 8;
+#pragma unroll
+            for (int it = 0; it < kRounds; ++it) qv[it] = tq[it] >= 0 ? ldg16(qbase + (long long)tq[it] * p.qs.t) : zero4;
+#pragma unroll
+            for (int it = 0; it < kRounds; ++it)
+                *reinterpret_cast<uint4*>(smem + kOffQ1 + swz(it * 8 + warp * 2 + sub, cc)) = qv[it];
+            fence_proxy_async();
+            mbar_arrive(bar_q);
+        }
+        __syncwarp();
+        const uint32_t tm_s = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's lanes: S / P
+        const uint32_t tm_o = tm_s + 128;                             // O
+        float m_ref = -INFINITY, l_run = 0.f;
+        for (int j = J0; j < J1; ++j) {
+            const int n = j - J0;
+            mbar_wait(bar_s, n & 1, abort_flag, p.wait_cycles, p.status, 30);
+            __syncwarp();
+            tc_fence_after();
+            softmax_tile(tm_s, tm_o, lo, hi, j * kTileN, p.scale_log2, n > 0, m_ref, l_run);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+        // ---- epilogue: O / l -> bf16 -> staged in the Q tile's shared memory -> the rows' token positions ----------
+        mbar_wait(bar_o, 0, abort_flag, p.wait_cycles, p.status, 40);
+        __syncwarp();
+        tc_fence_after();
+        const float inv = 1.f / l_run;
+        int* trow_s = reinterpret_cast<int*>(smem + kOffK1);          // the K slot is idle by now
+        trow_s[r] = t_row;
+        uint8_t* stage = smem + kOffQ1 + r * 256;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tm_o + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+                w.y = pack_bf16(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+                w.z = pack_bf16(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+                w.w = pack_bf16(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+                *reinterpret_cast<uint4*>(stage + (((c * 4 + v) ^ (r & 15)) << 4)) = w;
+            }
+        }
+        asm volatile("bar.sync 1, %0;" :: "n"(kTileM) : "memory");      // the 128 softmax threads
+        const int sub = r >> 4, l16 = r & 15;                           // 8 rows per pass
+#pragma unroll
+        for (int pass = 0; pass < kTileM / 8; ++pass) {
+            const int R = pass * 8 + sub, t_out = trow_s[R];
+            if (t_out >= 0)
+                *reinterpret_cast<uint4*>(Ob + (long long)t_out * p.os.t + l16 * 8) =
+                    *reinterpret_cast<const uint4*>(smem + kOffQ1 + R * 256 + ((l16 ^ (R & 15)) << 4));
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {   // a wait gave up: give copies and products still in flight time to land before leaving
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) { }
+        __syncthreads();
+    }
+    if (warp == kMmaWarp1) tmem_dealloc(tmem, kTmemCols1);
+}
+
 // ---- host side: tensor maps over the caller's K / V (two 64-column boxes of kTileN keys per tile) ---------
 bool make_kv_map(CUtensorMap* map, const void* base, const int64_t st[3], int B, int S, int H) {
     return make_bshd_map(map, base, st, B, S, H, 2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 64, kTileN, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -634,6 +886,11 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         if (cudaFuncGetAttributes(&fa, attention_tc_kernel<false>) != cudaSuccess || fa.numRegs != 168 ||
             cudaFuncGetAttributes(&fa, attention_tc_kernel<true>) != cudaSuccess || fa.numRegs != 168)
             return cudaErrorInvalidDeviceFunction;
+        // the single form: 256 threads at 128 registers, traded 128 x 200 + 128 x 56
+        e = cudaFuncSetAttribute(attention_tc_single_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes1);
+        if (e != cudaSuccess) return e;
+        if (cudaFuncGetAttributes(&fa, attention_tc_single_kernel) != cudaSuccess || fa.numRegs != kRegs1)
+            return cudaErrorInvalidDeviceFunction;
         attr_set = true;
     }
     TcParams tp{};
@@ -655,8 +912,9 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     const double ctas_shared = (double)s.batch * s.n_q_heads * ceil(s.seq * kept_frac / (kQTiles * kTileM));
     int sms = 148;
     { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
+    const bool single = ctx->attention_form == 3;
     const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 1.0 * sms);
-    const int rows_per_cta = split ? kTileM : kQTiles * kTileM;
+    const int rows_per_cta = (split || single) ? kTileM : kQTiles * kTileM;
     tp.n_row_blocks = (s.seq + rows_per_cta - 1) / rows_per_cta;
     {
         const long long kept_est = (p.select_mode == TF_SELECT_RATIO) ? (long long)s.seq - (long long)floor(p.prune_ratio * (double)s.seq)
@@ -669,10 +927,11 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     const long long n_ctas = (long long)tp.n_row_blocks * s.n_q_heads * s.batch;
     if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
     cudaError_t e;
-    if (split) e = launch_dependent(attention_tc_kernel<true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<true>::kSmemBytes, st, tp, mapK, mapV);
+    if (single) e = launch_dependent(attention_tc_single_kernel, dim3((unsigned)n_ctas), dim3(kThreads1), kSmemBytes1, st, tp, mapK, mapV);
+    else if (split) e = launch_dependent(attention_tc_kernel<true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<true>::kSmemBytes, st, tp, mapK, mapV);
     else       e = launch_dependent(attention_tc_kernel<false>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     ctx->launches += 1;
-    ctx->last_attention_kernel = split ? TF_KERNEL_ATTN_TC_SPLIT : TF_KERNEL_ATTN_TC_SHARED;
+    ctx->last_attention_kernel = single ? TF_KERNEL_ATTN_TC_SINGLE : (split ? TF_KERNEL_ATTN_TC_SPLIT : TF_KERNEL_ATTN_TC_SHARED);
     return e;
 }
 

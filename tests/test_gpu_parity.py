@@ -271,8 +271,9 @@ def test_select_few_candidates_left_with_ties_at_the_cut(S, n_tied):
 
 
 # ------------------------------------------------------------------------------- a5
-# path 2 / 3: the tensor-core kernel with K/V tiles shared by two Q tiles / split between the softmax groups
-@pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 1),
+# path 2 / 3 / 4: the tensor-core kernel with K/V tiles shared by two Q tiles / split between the softmax groups / one Q
+# tile and one softmax group per CTA, two CTAs per SM
+@pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 4), (torch.bfloat16, 1),
                                                 (torch.bfloat16, 0), (torch.float32, 0)])
 @pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5),
                                                     (1, 257, 8, 2, 0, 0.3), (2, 300, 4, 1, 64, 0.5),
@@ -304,12 +305,12 @@ def _assert_attention_kernel(ctx, dtype, path):
     if dtype != torch.bfloat16 or path == 0:
         assert ran == tfb.TF_KERNEL_ATTN_SIMT
     elif path == 1:
-        assert ran in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT)
+        assert ran in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT, tfb.TF_KERNEL_ATTN_TC_SINGLE)
     else:
-        assert ran == {2: tfb.TF_KERNEL_ATTN_TC_SHARED, 3: tfb.TF_KERNEL_ATTN_TC_SPLIT}[path]
+        assert ran == {2: tfb.TF_KERNEL_ATTN_TC_SHARED, 3: tfb.TF_KERNEL_ATTN_TC_SPLIT, 4: tfb.TF_KERNEL_ATTN_TC_SINGLE}[path]
 
 
-@pytest.mark.parametrize("dtype,path", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 0), (torch.float32, 0)])
+@pytest.mark.parametrize("dtype,path", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 4), (torch.bfloat16, 0), (torch.float32, 0)])
 @pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5), (1, 257, 8, 2, 0, 0.3),
                                                     (2, 300, 4, 1, 64, 0.5), (1, 515, 2, 2, 1, 0.7),
                                                     (1, 1300, 4, 2, 300, 0.5), (2, 1024, 2, 1, 0, 0.25)])
@@ -343,7 +344,7 @@ def test_layer_filter_retained_keys_only():
     assert n_mis == 0
 
 
-@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("path", [2, 3, 4])
 def test_pruned_attention_nothing_kept_and_everything_kept(path):
     q, k, v = _qkv(2, 70, 2, 2, torch.bfloat16)
     g = Gpu(q, k, v)
@@ -360,7 +361,7 @@ def test_pruned_attention_nothing_kept_and_everything_kept(path):
     g.close()
 
 
-@pytest.mark.parametrize("tensor_cores", [2, 3])
+@pytest.mark.parametrize("tensor_cores", [2, 3, 4])
 @pytest.mark.parametrize("claimed_ratio", [0.0, 0.9])
 def test_pruned_attention_with_a_retained_list_the_ratio_does_not_predict(tensor_cores, claimed_ratio):
     """tf_pruned_attention takes any retained list; the kernel orders its row blocks by the count the prune ratio
@@ -682,3 +683,43 @@ def test_decode_steps_match_oracle(dtype, mode, window, S0, T, Hq, Hkv):
     assert 0 < n_skips < B * T            # the case exercises both branches (skip and attend)
     assert near <= 2
     ctx.close()
+
+
+# ------------------------------------------------------------------------------- seeded random sweep
+@pytest.mark.parametrize("case", range(32))
+def test_layer_filter_random_shapes_modes_and_layouts(case):
+    """A seeded sweep over what the named cases do not pair up: shapes with ragged tiles, every anchor mode, fusion
+    mode and K/V visibility, windows, ratios, both dtypes and every attention form, each against the oracle."""
+    rng = np.random.default_rng(1000 + case)
+    dtype = torch.float32 if case % 8 == 7 else torch.bfloat16
+    B = int(rng.integers(1, 4))
+    S = int(rng.choice([1, 2, 17, 127, 128, 129, 255, 300, 513, 777, 1025, 1400]))
+    Hkv = int(rng.choice([1, 2, 3, 4, 8]))
+    Hq = Hkv * int(rng.choice([1, 2, 4]))
+    window = int(rng.choice([0, 0, 1, 37, 128, 400]))
+    ratio = float(rng.choice([0.0, 0.1, 0.3, 0.5, 0.7, 0.95]))
+    kw = dict(prune_ratio=ratio, warmup_tokens=int(rng.choice([1, 4, 9])),
+              anchor_mode=int(rng.choice([tfb.TF_ANCHOR_PAST_MEAN, tfb.TF_ANCHOR_INCL_MEAN, tfb.TF_ANCHOR_EMA])),
+              gamma=float(rng.choice([0.8, 0.9, 0.95])),
+              fuse_mode=int(rng.choice([tfb.TF_FUSE_INVVAR, tfb.TF_FUSE_EQ2_LITERAL, tfb.TF_FUSE_KEY_ONLY,
+                                        tfb.TF_FUSE_VALUE_ONLY, tfb.TF_FUSE_MEAN])),
+              kv_visibility=int(rng.choice([tfb.TF_KV_ALL, tfb.TF_KV_ALL, tfb.TF_KV_RETAINED])))
+    if kw["anchor_mode"] == tfb.TF_ANCHOR_INCL_MEAN:
+        kw["warmup_tokens"] = max(kw["warmup_tokens"], 1)
+    q, k, v = _qkv(B, S, Hq, Hkv, dtype, seed=2000 + case, dup=float(rng.choice([0.0, 0.25, 0.6])))
+    qn, kn, vn = oracle_inputs(q, k, v)
+    ref = oracle.layer_filter(qn, kn, vn, window=window, **kw)
+    g = Gpu(q, k, v, window=window, **kw)
+    g.ctx.tf_set_attention_path(int(rng.choice([1, 2, 3, 4])) if dtype == torch.bfloat16 else 0)
+    g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
+    g.status_ok()
+    assert np.abs(to_np(g.score) - ref["score"]).max() < SCORE_ATOL
+    n_mis, n_out = mask_disagreements(g.keep.cpu().numpy(), ref)
+    assert n_out == 0, f"{n_mis} keep/prune disagreements, {n_out} outside the 1e-6 band around theta"
+    if n_mis:      # compare the attention on the oracle's own retained list
+        g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, torch.from_numpy(ref["kept_idx"]).to(DEV),
+                                  torch.from_numpy(ref["n_kept"]).to(DEV), g.O)
+    o = to_np(g.O)
+    assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
+    assert np.all(o[ref["keep_mask"] == 0] == 0.0)
+    g.close()
