@@ -19,6 +19,7 @@ namespace tf {
 
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kMaxTableChunks = 64;   // longer sequences (> 65536 tokens) fall back to two block scans per 1024 tokens
 
 // Monotone map float -> uint32 (larger score <=> larger key); -0 and +0 share a key.
 __device__ __forceinline__ unsigned int score_key(float s) {
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
     __shared__ int s_warp[kSelWarps];
     __shared__ unsigned int s_prefix;
     __shared__ int s_rank, s_count, s_few_eq, s_total;
-    __shared__ int s_tab[KPT > 0 ? KPT : 1][kSelWarps];   // [chunk][warp] ballot counts of the final sweep
+    __shared__ int s_tab[KPT > 0 ? KPT : kMaxTableChunks][kSelWarps];   // [chunk][warp] ballot counts of the final sweep
     __shared__ unsigned int s_few[32];
 
     grid_launch_dependents();   // one CTA per sequence: the attention grid may take the other SMs and set up meanwhile
@@ -299,6 +300,77 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectPara
             const unsigned int bal = __ballot_sync(0xffffffffu, keep);
             const int pos = tab[i * kSelWarps + wid] + __popc(bal & lt);
             if (prune) th_min = fminf(th_min, sreg[i]);
+            if (in) {
+                p.keep_mask[(size_t)b * S + t] = keep ? 1 : 0;
+                if (keep) p.kept_idx[(size_t)b * S + pos] = t;
+            }
+        }
+        kept_base = s_total;
+    } else if ((S + kSelThreads - 1) / kSelThreads <= kMaxTableChunks) {
+        // The same one-scan-per-question sweep with a run-time number of chunks: the per-chunk decisions are kept as bits
+        // of two 64-bit words per thread, the scores are read again (shared or global memory) where they are needed.
+        const int n_chunks = (S + kSelThreads - 1) / kSelThreads;
+        int* tab = &s_tab[0][0];
+        const int lane = tid & 31, wid = tid >> 5;
+        const unsigned int lt = (1u << lane) - 1u;
+        auto scan_table = [&]() {          // exclusive prefix over tab[0 .. n_chunks*32), in place; s_total = the sum
+            __syncthreads();
+            if (wid == 0) {
+                int sum = 0;
+                for (int e = 0; e < n_chunks; ++e) sum += tab[lane * n_chunks + e];
+                int incl = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += n;
+                }
+                int run = incl - sum;
+                for (int e = 0; e < n_chunks; ++e) { const int v = tab[lane * n_chunks + e]; tab[lane * n_chunks + e] = run; run += v; }
+                if (lane == 31) s_total = incl;
+            }
+            __syncthreads();
+        };
+        unsigned long long eq_bits = 0ull, prune_bits = 0ull;
+        for (int i = 0; i < n_chunks; ++i) {
+            const int t = i * kSelThreads + tid;
+            const float sv = t < S ? sc[t] : 0.f;
+            const bool cand = t < S && candidate(t, sv);
+            if (p.mode == TF_SELECT_THRESHOLD) {
+                if (cand && sv > tau) prune_bits |= 1ull << i;
+            } else if (!nothing && cand) {
+                const unsigned int k = score_key(sv);
+                if (k > key_thr) prune_bits |= 1ull << i;
+                if (k == key_thr) eq_bits |= 1ull << i;
+            }
+        }
+        if (p.mode != TF_SELECT_THRESHOLD && !nothing) {      // CTA-uniform
+            for (int i = 0; i < n_chunks; ++i) {
+                const unsigned int bal = __ballot_sync(0xffffffffu, (eq_bits >> i) & 1ull);
+                if (lane == 0) tab[i * kSelWarps + wid] = __popc(bal);
+            }
+            scan_table();
+            for (int i = 0; i < n_chunks; ++i) {
+                const bool eq = (eq_bits >> i) & 1ull;
+                const unsigned int bal = __ballot_sync(0xffffffffu, eq);
+                const int eq_rank = tab[i * kSelWarps + wid] + __popc(bal & lt);     // 0-based among equals, index order
+                if (eq && eq_rank >= n_eq - take_eq) prune_bits |= 1ull << i;        // the take_eq equals with the highest index
+            }
+            __syncthreads();                                   // the table is reused below
+        }
+        for (int i = 0; i < n_chunks; ++i) {
+            const int t = i * kSelThreads + tid;
+            const bool keep = t < S && !((prune_bits >> i) & 1ull);
+            const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) tab[i * kSelWarps + wid] = __popc(bal);
+        }
+        scan_table();
+        for (int i = 0; i < n_chunks; ++i) {
+            const int t = i * kSelThreads + tid;
+            const bool in = t < S, prune = (prune_bits >> i) & 1ull;
+            const bool keep = in && !prune;
+            const unsigned int bal = __ballot_sync(0xffffffffu, keep);
+            const int pos = tab[i * kSelWarps + wid] + __popc(bal & lt);
+            if (prune) th_min = fminf(th_min, sc[t]);
             if (in) {
                 p.keep_mask[(size_t)b * S + t] = keep ? 1 : 0;
                 if (keep) p.kept_idx[(size_t)b * S + pos] = t;

@@ -224,7 +224,7 @@ def _select_case(score, ratio, warm, elig=None, mode=tfb.TF_SELECT_RATIO, thr=No
     g.close()
 
 
-@pytest.mark.parametrize("S", [1, 2, 31, 1024, 1025, 2048, 2049, 5000, 8193, 16384, 16385, 40000, 51200, 60000])   # register forms of 2, 4, 8, 16 scores per thread, then scores staged in shared memory (up to 51200), then re-read from global memory
+@pytest.mark.parametrize("S", [1, 2, 31, 1024, 1025, 2048, 2049, 5000, 8193, 16384, 16385, 40000, 51200, 60000, 70000])   # register forms of 2, 4, 8, 16 scores per thread, then scores staged in shared memory (up to 51200), then re-read from global memory (one-scan sweep up to 65536 tokens, block scans beyond)
 @pytest.mark.parametrize("ratio", [0.0, 0.25, 0.5, 0.7, 0.999])
 def test_select_bit_exact_random(S, ratio):
     rng = np.random.default_rng(S)
