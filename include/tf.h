@@ -18,7 +18,9 @@
  *   - every tensor pointer is DEVICE memory owned by the caller; the library reads its
  *     inputs, writes its outputs, keeps no pointer after the call returns;
  *   - calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*,
- *     NULL = default stream), do not synchronise and do not allocate;
+ *     NULL = default stream), do not synchronise and do not allocate; after one call of the
+ *     same shape outside a capture (it clears the scratch and sets function attributes) a call
+ *     may be captured into a CUDA graph and replayed: nothing about a launch lives on the host;
  *   - the return value reports host-side validation and launch errors only; conditions
  *     found on the device (a bounded wait that gave up) are read with tf_get_status;
  *   - head_dim must be 128; Q/K/V/O rows (head_dim elements) are contiguous and 16-byte

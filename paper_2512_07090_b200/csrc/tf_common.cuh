@@ -129,26 +129,36 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 
 namespace tf {
 // Host-side bookkeeping of one scan scratch region (the first section of a workspace).
-// The region starts with two counter words {ticket, finished}: every CTA (or worker) of a scan launch draws its
-// work from `ticket`, and the last CTA to leave the kernel sets both words back to zero, so a launch always starts
-// counting at zero whatever happened to the launch before it (a wait that gave up, workers that stopped drawing).
+// The region starts with three counter words {ticket, finished, launches}: every CTA (or worker) of a scan launch
+// draws its work from `ticket`; the last CTA to leave the kernel sets ticket and finished back to zero, so a launch
+// always starts counting at zero whatever happened to the launch before it (a wait that gave up, workers that stopped
+// drawing), and advances `launches`, from which the next launch derives the tag that marks its records as its own.
+// Nothing about a launch lives on the host, so a captured launch can be replayed (CUDA graphs) with fresh tags.
 struct ScanScratch {
     void* ptr = nullptr;
     size_t capacity = 0;            // bytes the owner of the region provides
     size_t bytes = 0;               // layout key of the records cleared last (0: never cleared)
-    unsigned int epoch = 0;         // tag of the latest launch
     bool needs_clear = true;
 };
 constexpr size_t kScanCounterBytes = 256;   // {ticket, finished} + padding in front of the records
 
+// The tag of this launch's records (never 0, the tag of cleared memory).  Read by every thread that needs it after
+// grid_dependency_wait() and BEFORE its CTA calls scan_leave (the last CTA to leave advances the word).
+__device__ __forceinline__ unsigned int scan_launch_tag(const unsigned int* counters) {
+    const unsigned int n = *reinterpret_cast<const volatile unsigned int*>(counters + 2);
+    return n == 0xffffffffu ? 1u : n + 1u;
+}
 // Drawn by one thread per CTA / worker after grid_dependency_wait().
 __device__ __forceinline__ unsigned int scan_draw_ticket(unsigned int* counters) { return atomicAdd(counters, 1u); }
-// Called by one thread per CTA when the CTA will draw no more tickets; n_ctas = gridDim.x.
+// Called by one thread per CTA when the CTA will draw no more tickets (and its threads have read the launch tag);
+// n_ctas = gridDim.x.
 __device__ __forceinline__ void scan_leave(unsigned int* counters, unsigned int n_ctas) {
     __threadfence();
     if (atomicAdd(counters + 1, 1u) == n_ctas - 1u) {
         atomicExch(counters, 0u);
         atomicExch(counters + 1, 0u);
+        const unsigned int n = *reinterpret_cast<volatile unsigned int*>(counters + 2);
+        atomicExch(counters + 2, n == 0xffffffffu ? 1u : n + 1u);
     }
 }
 }  // namespace tf

@@ -10,7 +10,7 @@
 //   - chunk c takes P of the nearest earlier anchor chunk a and adds the aggregates a..c-1 in
 //     ascending order.  The association is fixed, so results do not depend on timing.
 // A record is 128 16-byte packets {k value, v value, tag, 0}; a packet is valid when its tag is
-// this launch's epoch, so value and validity arrive in one load and nothing is cleared between
+// this launch's tag (derived from a launch counter in the scratch itself), so value and validity arrive in one load and nothing is cleared between
 // launches.  Tiles are handed out by an atomic ticket, chunk index slowest, so every record a
 // running tile waits for belongs to a tile that has itself started: the waits cannot deadlock,
 // and every wait is bounded anyway (on expiry the kernel records TF_ERR_TIMEOUT and goes on).
@@ -45,8 +45,8 @@ struct ScanParams {
     const float* sum_k_in; const float* sum_v_in; const long long* count_in;
     float* sum_k_out; float* sum_v_out;
     float* sim_k; float* sim_v;
-    unsigned int* counters;   // {ticket, finished}: see ScanScratch
-    unsigned int epoch, n_tiles;
+    unsigned int* counters;   // {ticket, finished, launches}: see ScanScratch
+    unsigned int n_tiles;
     uint4* agg_rec;      // [tile][128] packets, tile = chunk * n_chains + chain
     uint4* prefix_rec;   // [(chunk / kAnchorEvery) * n_chains + chain][128] packets
     DevStatus* status;
@@ -94,15 +94,16 @@ __global__ void __launch_bounds__(kScanThreads, 4) kv_stats_kernel(const ScanPar
     constexpr int NV = Elem<T>::kVecPerLane, EPV = Elem<T>::kPerVec;
 
     __shared__ __align__(16) float sub[2][kGroups][kHeadDim];
-    __shared__ unsigned int s_ticket;
+    __shared__ unsigned int s_ticket, s_tag;
 
     const int tid = threadIdx.x, g = tid >> 3, l = tid & 7;
     if (tid == 0) {
+        s_tag = scan_launch_tag(p.counters);
         s_ticket = scan_draw_ticket(p.counters);
         scan_leave(p.counters, gridDim.x);        // one ticket per CTA: this CTA draws no more
     }
     __syncthreads();
-    const unsigned int tile = s_ticket;
+    const unsigned int tile = s_ticket, epoch = s_tag;
     if (tile >= p.n_tiles) return;                // cannot happen while the counters are intact; never index records with it
     const int c = (int)(tile / (unsigned)p.n_chains), chain = (int)(tile % (unsigned)p.n_chains);
     const int b = chain / p.H, h = chain % p.H;
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(kScanThreads, 4) kv_stats_kernel(const ScanPar
     }
 
     // every chunk but the last of its chain publishes its aggregate
-    if (c + 1 < p.n_chunks) st_packet(p.agg_rec + (size_t)tile * kHeadDim + tid, agg_k, agg_v, p.epoch);
+    if (c + 1 < p.n_chunks) st_packet(p.agg_rec + (size_t)tile * kHeadDim + tid, agg_k, agg_v, epoch);
 
     float carry_k = 0.f, carry_v = 0.f;
     if (c == 0) {
@@ -200,19 +201,19 @@ __global__ void __launch_bounds__(kScanThreads, 4) kv_stats_kernel(const ScanPar
             for (int u = 0; u < kPollBatch; ++u) {
                 if (j0 + u < c) {
                     r[u] = wait_packet(p.agg_rec + ((size_t)(j0 + u) * p.n_chains + chain) * kHeadDim + tid, r[u],
-                                       p.epoch, p.max_polls, p.status, tile);
+                                       epoch, p.max_polls, p.status, tile);
                     Ak = EMA ? fmaf(a_full, Ak, __uint_as_float(r[u].x)) : Ak + __uint_as_float(r[u].x);
                     Av = EMA ? fmaf(a_full, Av, __uint_as_float(r[u].y)) : Av + __uint_as_float(r[u].y);
                     decay_to_here *= a_full;
                 }
             }
         }
-        pfirst = wait_packet(prec, pfirst, p.epoch, p.max_polls, p.status, tile);
+        pfirst = wait_packet(prec, pfirst, epoch, p.max_polls, p.status, tile);
         carry_k = EMA ? fmaf(decay_to_here, __uint_as_float(pfirst.x), Ak) : __uint_as_float(pfirst.x) + Ak;
         carry_v = EMA ? fmaf(decay_to_here, __uint_as_float(pfirst.y), Av) : __uint_as_float(pfirst.y) + Av;
     }
     if (c % kAnchorEvery == 0 && c + 1 < p.n_chunks)
-        st_packet(p.prefix_rec + ((size_t)(c / kAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, p.epoch);
+        st_packet(p.prefix_rec + ((size_t)(c / kAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry_k, carry_v, epoch);
     if (c + 1 == p.n_chunks) {
         if (p.sum_k_out) p.sum_k_out[(size_t)chain * kHeadDim + tid] = fmaf(a_chunk, carry_k, agg_k);
         if (p.sum_v_out) p.sum_v_out[(size_t)chain * kHeadDim + tid] = fmaf(a_chunk, carry_v, agg_v);
@@ -324,14 +325,12 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
     // The region is also cleared when its extent changes: another shape's layout may have put
     // other data where this shape keeps records.
     if (ws->capacity < pl.bytes) return cudaErrorInvalidValue;
-    if (ws->needs_clear || ws->bytes != pl.bytes || ws->epoch == 0xffffffffu) {
+    if (ws->needs_clear || ws->bytes != pl.bytes) {
         cudaError_t e = cudaMemsetAsync(ws->ptr, 0, pl.bytes, st);
         if (e != cudaSuccess) return e;
         ws->needs_clear = false;
         ws->bytes = pl.bytes;
-        ws->epoch = 0;
     }
-    ws->epoch += 1;
 
     ScanParams sp{};
     sp.K = K; sp.V = V;
@@ -350,7 +349,6 @@ cudaError_t launch_kv_stats(tf_ctx* ctx, const tf_shape& s, const tf_filter_para
     sp.sim_k = sim_k; sp.sim_v = sim_v;
     char* base = static_cast<char*>(ws->ptr);
     sp.counters = reinterpret_cast<unsigned int*>(base);
-    sp.epoch = ws->epoch;
     sp.n_tiles = (unsigned int)tiles;
     sp.agg_rec = reinterpret_cast<uint4*>(base + pl.agg_offset);
     sp.prefix_rec = reinterpret_cast<uint4*>(base + pl.prefix_offset);

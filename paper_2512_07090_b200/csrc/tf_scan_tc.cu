@@ -205,7 +205,6 @@ struct Gram1Params {
     const float* sum_in[2]; const long long* count_in;
     float* sum_out[2];
     float* sim[2];
-    unsigned int epoch;
     uint2* agg_rec[2]; uint2* prefix_rec[2];
     DevStatus* status;
     int max_polls;               // bounded waits: polls of one look-back packet ...
@@ -259,6 +258,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
     // Work goes by ticket, chunk index slowest (K and V of a tile side by side): the records a tile waits for belong
     // to tickets drawn before its own, by CTAs that are running, whatever order the CTAs were started in.
     if (tid == 0) {
+        s_ticket[1] = scan_launch_tag(p.counters);
         const unsigned int t = scan_draw_ticket(p.counters);
         scan_leave(p.counters, gridDim.x);     // one ticket per CTA
         *s_ticket = t;
@@ -272,7 +272,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
         }
     }
     __syncthreads();
-    const unsigned int ticket = *s_ticket;
+    const unsigned int ticket = s_ticket[0], epoch = s_ticket[1];
     if (ticket >= p.n_work) {                  // cannot happen while the counters are intact; never index records with it
         tc_fence_before();
         __syncthreads();
@@ -332,7 +332,7 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
         tmem_wait_ld();
         agg = an.agg_of(r0) + an.agg_of(r1);
     }
-    if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, p.epoch);
+    if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, epoch);
     tc_fence_before();
     __syncthreads();
 
@@ -346,11 +346,11 @@ kv_stats_gram1_kernel(const Gram1Params p, const __grid_constant__ CUtensorMap m
             float A = 0.f;
 #pragma unroll
             for (int u = 0; u < kGramAnchorEvery; ++u)       // requested while the tile was in flight
-                if (a0 + u < c) A = an.look_back(A, wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile));
-            carry = an.carry_of(wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile), A, c - a0);
+                if (a0 + u < c) A = an.look_back(A, wait_packet2(arec + u * astride, afirst[u], epoch, p.max_polls, p.status, tile));
+            carry = an.carry_of(wait_packet2(prec, pfirst, epoch, p.max_polls, p.status, tile), A, c - a0);
         }
         if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
-            st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, p.epoch);
+            st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, epoch);
         if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = an.sum_after(carry, agg, valid);
     };
     const bool publishes_prefix = (c % kGramAnchorEvery == 0);
@@ -589,6 +589,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
     };
 
     grid_dependency_wait();   // the set-up above overlaps the tail of the kernel before this one on the stream
+    const unsigned int epoch = scan_launch_tag(p.counters);
     if (tid == 0) announce_and_load(draw());
     worker_sync(w);
     uint4 cur = make_uint4(s_next[0], s_next[1], s_next[2], s_next[3]);
@@ -643,7 +644,7 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             tmem_wait_ld();
             agg = an.agg_of(r0);
         }
-        if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, p.epoch);
+        if (c + 1 < p.n_chunks) st_packet2(agg_rec + (size_t)tile * kHeadDim + tid, agg, epoch);
 
         // ---- carry: prefix record of chunk a0 + aggregates of chunks a0 .. c-1, in ascending order ---------------------
         float carry = 0.f;
@@ -653,11 +654,11 @@ kv_stats_gram_persistent_kernel(const GramPParams pp, const __grid_constant__ CU
             float A = 0.f;
 #pragma unroll
             for (int u = 0; u <= kPLookBack; ++u)
-                if (a0 + u < c) A = an.look_back(A, wait_packet2(arec + u * astride, afirst[u], p.epoch, p.max_polls, p.status, tile));
-            carry = an.carry_of(wait_packet2(prec, pfirst, p.epoch, p.max_polls, p.status, tile), A, c - a0);
+                if (a0 + u < c) A = an.look_back(A, wait_packet2(arec + u * astride, afirst[u], epoch, p.max_polls, p.status, tile));
+            carry = an.carry_of(wait_packet2(prec, pfirst, epoch, p.max_polls, p.status, tile), A, c - a0);
         }
         if (c % kGramAnchorEvery == 0 && c + 1 < p.n_chunks)
-            st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, p.epoch);
+            st_packet2(prefix_rec + ((size_t)(c / kGramAnchorEvery) * p.n_chains + chain) * kHeadDim + tid, carry, epoch);
         if (c + 1 == p.n_chunks && p.sum_out[x]) p.sum_out[x][(size_t)chain * kHeadDim + tid] = an.sum_after(carry, agg, valid);
         {   // the carry as c1 + c2 + c3 (bf16 each) into rows 0-2 of the small operand
             float cr = carry;
@@ -778,14 +779,12 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
         return cudaErrorNotSupported;
     // (the low bit of the layout key distinguishes this record layout from the plain kernel's, which may share the scratch)
     const size_t key = gl.bytes | 1;
-    if (ws->needs_clear || ws->bytes != key || ws->epoch == 0xffffffffu) {
+    if (ws->needs_clear || ws->bytes != key) {
         cudaError_t e = cudaMemsetAsync(ws->ptr, 0, gl.bytes, st);
         if (e != cudaSuccess) return e;
         ws->needs_clear = false;
         ws->bytes = key;
-        ws->epoch = 0;
     }
-    ws->epoch += 1;
 
     static bool attr_set_dev[kDeviceFlagSlots] = {};      // function attributes are per device
     bool& attr_set = attr_set_dev[ctx->device >= 0 && ctx->device < kDeviceFlagSlots ? ctx->device : 0];
@@ -807,7 +806,6 @@ cudaError_t launch_kv_stats_gram(tf_ctx* ctx, const tf_shape& s, const tf_filter
     }
     gp.sim[0] = sim_k; gp.sim[1] = sim_v;
     char* base = static_cast<char*>(ws->ptr);
-    gp.epoch = ws->epoch;
     const size_t rec = kHeadDim * sizeof(uint2);
     for (int x = 0; x < 2; ++x) {
         gp.agg_rec[x] = reinterpret_cast<uint2*>(base + gl.agg_offset + x * tiles * rec);

@@ -723,3 +723,39 @@ def test_layer_filter_random_shapes_modes_and_layouts(case):
     assert attn_rel_err(o, ref["O"]) < ATTN_TOL[dtype]
     assert np.all(o[ref["keep_mask"] == 0] == 0.0)
     g.close()
+
+
+def test_layer_filter_replayed_from_a_cuda_graph_with_new_inputs():
+    """One tf_layer_filter call captured into a CUDA graph (after a first call outside the capture, which clears the
+    scratch and sets function attributes) and replayed over buffers whose contents change between replays: everything a
+    launch needs to tell its own look-back records from an earlier launch's lives on the device, so every replay is
+    right.  Both Gram-scan kernels and the CUDA-core scan."""
+    B, S, Hq, Hkv = 2, 1300, 8, 2
+    inputs = [_qkv(B, S, Hq, Hkv, torch.bfloat16, seed=90 + i) for i in range(3)]
+    for scan_path in (2, 3, 1):
+        q, k, v = (t.clone() for t in inputs[0])
+        g = Gpu(q, k, v, prune_ratio=0.5, warmup_tokens=4)
+        g.ctx.tf_set_scan_path(scan_path)
+        g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)     # outside the capture
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
+        torch.cuda.current_stream().wait_stream(side)
+        for qi, ki, vi in inputs[1:] + inputs[:1]:
+            q.copy_(qi); k.copy_(ki); v.copy_(vi)
+            g.O.fill_(float("nan")); g.score.fill_(float("nan"))
+            graph.replay()
+            torch.cuda.synchronize()
+            g.status_ok()
+            qn, kn, vn = oracle_inputs(q, k, v)
+            ref = oracle.layer_filter(qn, kn, vn, prune_ratio=0.5, warmup_tokens=4)
+            assert np.abs(to_np(g.score) - ref["score"]).max() < SCORE_ATOL
+            n_mis, n_out = mask_disagreements(g.keep.cpu().numpy(), ref)
+            assert n_out == 0
+            if n_mis == 0:
+                assert attn_rel_err(to_np(g.O), ref["O"]) < ATTN_TOL[torch.bfloat16]
+        g.close()
