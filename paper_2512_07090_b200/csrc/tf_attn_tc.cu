@@ -198,10 +198,16 @@ __device__ __forceinline__ void softmax_tile(uint32_t tm_s, uint32_t tm_o, int l
     l_run = fmaf(l_run, corr, psum);
 }
 
-template <bool kSplit>
+template <bool kSplit, bool kHeads = false>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
+    static_assert(!(kSplit && kHeads), "the head-pair form is a variant of the shared form");
     using C = Cfg<kSplit>;
+    // retained-list entries one CTA covers; kOneSpan: both softmax groups work on the SAME 128 entries (the split form:
+    // alternate K/V tiles; the head-pair form: two query heads of one KV group, so that the groups' K/V tile ranges and
+    // masks coincide and no tile is ever worked on by one group alone)
+    constexpr bool kOneSpan = kSplit || kHeads;
+    constexpr int kRows = kOneSpan ? kTileM : C::kRows;
     constexpr int kStages = C::kStages, kOffQ = C::kOffQ, kOffRing = C::kOffRing, kOffBar = C::kOffBar, kStep = C::kStep;
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -240,16 +246,18 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     // instead of delaying the first wave of real work.  Any estimate gives a one-to-one assignment.
     int pair = p.first_pair - rb;
     if (pair < 0) pair += p.n_row_blocks;
-    const int qh = bh % p.Hq, b = bh / p.Hq;
+    constexpr int kHeadsPerCta = kHeads ? 2 : 1;
+    const int qh = (bh % (p.Hq / kHeadsPerCta)) * kHeadsPerCta, b = bh / (p.Hq / kHeadsPerCta);   // first (or only) head
     const int nk = p.n_kept[b];
-    const int slot0 = pair * C::kRows;
+    const int slot0 = pair * kRows;
     const int32_t* kept = p.kept_idx + (size_t)b * p.S;
     __nv_bfloat16* Ob = p.O + (long long)b * p.os.b + (long long)qh * p.os.h;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     if (slot0 >= max(nk, 1) || nk == 0) {   // no retained row in this block (CTA-uniform)
         if (slot0 < max(nk, 1)) {           // nothing retained at all: the whole head is zero
-            for (int i = tid; i < p.S * 16; i += kThreads)
-                *reinterpret_cast<uint4*>(Ob + (long long)(i >> 4) * p.os.t + (i & 15) * 8) = zero4;
+            for (int hh = 0; hh < kHeadsPerCta; ++hh)
+                for (int i = tid; i < p.S * 16; i += kThreads)
+                    *reinterpret_cast<uint4*>(Ob + (long long)hh * p.os.h + (long long)(i >> 4) * p.os.t + (i & 15) * 8) = zero4;
         }
         tc_fence_before();
         __syncthreads();
@@ -261,16 +269,17 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     // The softmax threads read the retained indices of the Q rows they will gather (16 lanes per 256-byte row, the
     // 8 warps take 16 rows per round) and of their own row now, next to the loads the set-up below waits for anyway:
     // one global round trip less between the set-up and the first Q K^T.
-    constexpr int kRounds = C::kRows / 16;
+    constexpr int kRounds = C::kRows / 16;   // 16 rows per round over the CTA's Q tiles
     int tq[kRounds];
     int t_row = -1;
     if (warp < kMmaWarp) {
 #pragma unroll
         for (int it = 0; it < kRounds; ++it) {
-            const int s_q = slot0 + it * 16 + warp * 2 + (lane >> 4);
+            const int rr = it * 16 + warp * 2 + (lane >> 4);           // row of the CTA's Q buffer (tile rr / 128)
+            const int s_q = slot0 + (kHeads ? (rr & (kTileM - 1)) : rr);
             tq[it] = s_q < nk ? kept[s_q] : -1;
         }
-        const int slot_pre = slot0 + (kSplit ? 0 : (warp >> 2) * kTileM) + (tid & (kTileM - 1));
+        const int slot_pre = slot0 + (kOneSpan ? 0 : (warp >> 2) * kTileM) + (tid & (kTileM - 1));
         if (slot_pre < nk) t_row = kept[slot_pre];
     }
 
@@ -279,7 +288,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     int jb[kQTiles], je[kQTiles];
 #pragma unroll
     for (int i = 0; i < kQTiles; ++i) {
-        const int s_lo = slot0 + (kSplit ? 0 : i * kTileM);
+        const int s_lo = slot0 + (kOneSpan ? 0 : i * kTileM);
         if (s_lo < nk) {
             const int s_last = min(s_lo + kTileM, nk) - 1;
             const int t_first = kept[s_lo], t_last = kept[s_last];
@@ -313,12 +322,15 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         // rows of pruned tokens that precede a retained row of this CTA (and follow the last retained
         // one) are zero; 16 lanes write one row
         const int g4 = (tid - (kTmaWarp + 1) * 32) >> 4, l16 = tid & 15;
-        const int s_end = min(slot0 + C::kRows, nk);
+        const int s_end = min(slot0 + kRows, nk);
         for (int s_z = slot0 + g4; s_z < s_end; s_z += 4) {
             const int prev = s_z == 0 ? -1 : kept[s_z - 1], cur = kept[s_z];
-            for (int t = prev + 1; t < cur; ++t) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + l16 * 8) = zero4;
-            if (s_z == nk - 1)
-                for (int t = cur + 1; t < p.S; ++t) *reinterpret_cast<uint4*>(Ob + (long long)t * p.os.t + l16 * 8) = zero4;
+            for (int hh = 0; hh < kHeadsPerCta; ++hh) {
+                __nv_bfloat16* Oz = Ob + (long long)hh * p.os.h + l16 * 8;
+                for (int t = prev + 1; t < cur; ++t) *reinterpret_cast<uint4*>(Oz + (long long)t * p.os.t) = zero4;
+                if (s_z == nk - 1)
+                    for (int t = cur + 1; t < p.S; ++t) *reinterpret_cast<uint4*>(Oz + (long long)t * p.os.t) = zero4;
+            }
         }
     } else if (warp == kTmaWarp) {
         // ================================ TMA producer ================================================
@@ -418,7 +430,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         const int i = warp >> 2;                 // group: its Q tile (shared) or its half of the K/V tiles (split)
         const int r = tid & (kTileM - 1);        // row within the tile
-        const int slot = slot0 + (kSplit ? 0 : i * kTileM) + r;
+        const int slot = slot0 + (kOneSpan ? 0 : i * kTileM) + r;
         const bool valid = slot < nk;               // t_row (fetched above) is the row's token position, -1 if none
         int hi = t_row;                                                           // visible keys: lo .. hi
         int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
@@ -432,7 +444,8 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             uint4 qv[kRounds];
             const __nv_bfloat16* qbase = p.Q + (long long)b * p.qs.b + (long long)qh * p.qs.h + cc * 8;
 #pragma unroll
-            for (int it = 0; it < kRounds; ++it) qv[it] = tq[it] >= 0 ? ldg16(qbase + (long long)tq[it] * p.qs.t) : zero4;
+            for (int it = 0; it < kRounds; ++it)   // head-pair form: rounds 8..15 fill the second head's tile
+                qv[it] = tq[it] >= 0 ? ldg16(qbase + (kHeads ? (long long)(it >> 3) * p.qs.h : 0ll) + (long long)tq[it] * p.qs.t) : zero4;
 #pragma unroll
             for (int it = 0; it < kRounds; ++it) {
                 const int rr = it * 16 + w8 * 2 + sub;
@@ -517,6 +530,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             __syncwarp();
             tc_fence_after();
             const float inv = 1.f / l_run;
+            __nv_bfloat16* Oi = Ob + (kHeads ? (long long)i * p.os.h : 0ll);   // this group's head
             int* trow_s = reinterpret_cast<int*>(smem + kOffRing + 4096) + i * kTileM;
             trow_s[r] = t_row;
             uint8_t* stage = smem + kOffQ + i * kTileBytes + r * 256;
@@ -541,7 +555,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             for (int pass = 0; pass < kTileM / 8; ++pass) {
                 const int R = pass * 8 + sub, t_out = trow_s[R];
                 if (t_out >= 0)
-                    *reinterpret_cast<uint4*>(Ob + (long long)t_out * p.os.t + l16 * 8) =
+                    *reinterpret_cast<uint4*>(Oi + (long long)t_out * p.os.t + l16 * 8) =
                         *reinterpret_cast<const uint4*>(smem + kOffQ + i * kTileBytes + R * 256 + ((l16 ^ (R & 15)) << 4));
             }
         }
@@ -873,6 +887,9 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg<false>::kSmemBytes);
         if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg<false>::kSmemBytes);
+        if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Cfg<true>::kSmemBytes);
         if (e != cudaSuccess) return e;
@@ -884,6 +901,7 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         // never answered by running another kernel.
         cudaFuncAttributes fa{};
         if (cudaFuncGetAttributes(&fa, attention_tc_kernel<false>) != cudaSuccess || fa.numRegs != 168 ||
+            cudaFuncGetAttributes(&fa, attention_tc_kernel<false, true>) != cudaSuccess || fa.numRegs != 168 ||
             cudaFuncGetAttributes(&fa, attention_tc_kernel<true>) != cudaSuccess || fa.numRegs != 168)
             return cudaErrorInvalidDeviceFunction;
         // the single form: 256 threads at 128 registers, traded 128 x 200 + 128 x 56
@@ -914,7 +932,12 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     { int dev = 0; if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); }
     const bool single = ctx->attention_form == 3;
     const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 1.0 * sms);
-    const int rows_per_cta = (split || single) ? kTileM : kQTiles * kTileM;
+    // Grouped-query attention with an even number of query heads per KV head: the two Q tiles of a shared-form CTA are
+    // the same 128 retained rows of two query heads of one group instead of 256 rows of one head.
+    const bool can_pair_heads = s.n_kv_heads > 0 && s.n_q_heads % s.n_kv_heads == 0 && (s.n_q_heads / s.n_kv_heads) % 2 == 0;
+    if (ctx->attention_form == 4 && !can_pair_heads) return cudaErrorNotSupported;
+    const bool heads = ctx->attention_form == 4 || (ctx->attention_form == 0 && !split && can_pair_heads);
+    const int rows_per_cta = (split || single || heads) ? kTileM : kQTiles * kTileM;
     tp.n_row_blocks = (s.seq + rows_per_cta - 1) / rows_per_cta;
     {
         const long long kept_est = (p.select_mode == TF_SELECT_RATIO) ? (long long)s.seq - (long long)floor(p.prune_ratio * (double)s.seq)
@@ -924,14 +947,16 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     }
     const double kv_bytes = 2.0 * s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
     tp.heads_fastest = (kv_bytes <= 48e6 || ctas_shared < 6.0 * sms) ? 1 : 0;   // K and V stay in L2, or balance matters more
-    const long long n_ctas = (long long)tp.n_row_blocks * s.n_q_heads * s.batch;
+    const long long n_ctas = (long long)tp.n_row_blocks * (heads ? s.n_q_heads / 2 : s.n_q_heads) * s.batch;
     if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
     cudaError_t e;
     if (single) e = launch_dependent(attention_tc_single_kernel, dim3((unsigned)n_ctas), dim3(kThreads1), kSmemBytes1, st, tp, mapK, mapV);
+    else if (heads) e = launch_dependent(attention_tc_kernel<false, true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     else if (split) e = launch_dependent(attention_tc_kernel<true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<true>::kSmemBytes, st, tp, mapK, mapV);
     else       e = launch_dependent(attention_tc_kernel<false>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     ctx->launches += 1;
-    ctx->last_attention_kernel = single ? TF_KERNEL_ATTN_TC_SINGLE : (split ? TF_KERNEL_ATTN_TC_SPLIT : TF_KERNEL_ATTN_TC_SHARED);
+    ctx->last_attention_kernel = single ? TF_KERNEL_ATTN_TC_SINGLE : heads ? TF_KERNEL_ATTN_TC_HEAD_PAIR
+                                        : split ? TF_KERNEL_ATTN_TC_SPLIT : TF_KERNEL_ATTN_TC_SHARED;
     return e;
 }
 
