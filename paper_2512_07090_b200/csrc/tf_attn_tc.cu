@@ -2,7 +2,9 @@
 // retained tokens only, head_dim 128.
 //
 // One CTA owns 256 consecutive entries of a sequence's retained list for one query head, as two
-// 128-row Q tiles that share every K/V tile.  Warp roles:
+// 128-row Q tiles that share every K/V tile -- or, on grouped-query shapes, the same 128 entries for
+// two query heads of one KV group (then both tiles need the same K/V tiles with the same masks).
+// Warp roles:
 //   warps 0-3 / 4-7  softmax group of Q tile 0 / 1 (thread r owns row r of its tile)
 //   warp 8           issues every tcgen05.mma (one lane)
 //   warp 9           TMA producer: K and V tiles of 128 keys into a 4-slot ring (one lane)
