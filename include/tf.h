@@ -255,7 +255,8 @@ enum { TF_KERNEL_NONE = 0,
        TF_KERNEL_ATTN_TC_SHARED = 11,       /* tcgen05 attention, two Q tiles share every K/V tile    */
        TF_KERNEL_ATTN_TC_SPLIT = 12,        /* tcgen05 attention, one Q tile, K/V tiles split         */
        TF_KERNEL_ATTN_TC_SINGLE = 13,       /* tcgen05 attention, one Q tile and one softmax group, two CTAs per SM */
-       TF_KERNEL_ATTN_TC_HEAD_PAIR = 14 };  /* tcgen05 attention, the same 128 rows of two query heads of one KV group share every K/V tile */
+       TF_KERNEL_ATTN_TC_HEAD_PAIR = 14,    /* tcgen05 attention, the same 128 rows of two query heads of one KV group share every K/V tile */
+       TF_KERNEL_ATTN_TC_HEAD_QUAD = 15 };  /* tcgen05 attention, the same 64 rows of four query heads of one KV group share every K/V tile */
 tf_status tf_last_kernels(tf_ctx *ctx, int32_t kernels[2]);
 
 /* Which attention kernel a bf16 call uses: 1 = tcgen05 tensor-core kernel (default; it picks between
@@ -264,7 +265,9 @@ tf_status tf_last_kernels(tf_ctx *ctx, int32_t kernels[2]);
  * kernel, two Q tiles per CTA sharing every K/V tile, 3 = tensor-core kernel, one Q tile per CTA with its
  * K/V tiles split between the CTA's two softmax groups, 4 = tensor-core kernel, one Q tile and one softmax group
  * per CTA, two CTAs per SM, 5 = tensor-core kernel, two query heads of one KV group per CTA (the same 128 retained
- * rows of both; needs an even number of query heads per KV head).  With 2, 3, 4 or 5 the named kernel is a requirement:
+ * rows of both; needs an even number of query heads per KV head), 6 = tensor-core kernel, four query heads of one KV group
+ * per CTA (the same 64 retained rows of all four; needs a multiple of four query heads per KV head).  With 2 to 6 the named
+ * kernel is a requirement:
  * a call it cannot take fails with TF_ERR_UNSUPPORTED instead of running another kernel.  For A/B checks. */
 tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
 

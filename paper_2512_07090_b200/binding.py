@@ -26,7 +26,7 @@ TF_KV_ALL, TF_KV_RETAINED = 0, 1
 TF_STATIC_SCRATCH_BYTES = 8 << 20
 (TF_KERNEL_NONE, TF_KERNEL_SCAN_PLAIN, TF_KERNEL_SCAN_GRAM_TILE, TF_KERNEL_SCAN_GRAM_PERSISTENT) = range(4)
 TF_KERNEL_ATTN_SIMT, TF_KERNEL_ATTN_TC_SHARED, TF_KERNEL_ATTN_TC_SPLIT, TF_KERNEL_ATTN_TC_SINGLE = 10, 11, 12, 13
-TF_KERNEL_ATTN_TC_HEAD_PAIR = 14
+TF_KERNEL_ATTN_TC_HEAD_PAIR, TF_KERNEL_ATTN_TC_HEAD_QUAD = 14, 15
 
 EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes", "tf_set_workspace",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",

@@ -501,7 +501,7 @@ tf_status tf_set_wait_limits(tf_ctx* ctx, int64_t max_polls, int64_t wait_cycles
 
 tf_status tf_set_attention_path(tf_ctx* ctx, int use_tensor_cores) {
     if (!ctx) return TF_ERR_INVALID_ARG;
-    if (use_tensor_cores < 0 || use_tensor_cores > 5) return TF_ERR_INVALID_ARG;
+    if (use_tensor_cores < 0 || use_tensor_cores > 6) return TF_ERR_INVALID_ARG;
     ctx->use_tensor_cores = use_tensor_cores ? 1 : 0;
     ctx->attention_form = use_tensor_cores >= 2 ? use_tensor_cores - 1 : 0;
     return TF_OK;

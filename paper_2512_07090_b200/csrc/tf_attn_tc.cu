@@ -200,16 +200,22 @@ __device__ __forceinline__ void softmax_tile(uint32_t tm_s, uint32_t tm_o, int l
     l_run = fmaf(l_run, corr, psum);
 }
 
-template <bool kSplit, bool kHeads = false>
+// kHpt = query heads per Q tile: 0 = the forms above (one head per CTA); 1, 2 = the head forms of the shared form for
+// grouped-query shapes: a Q tile holds the same 128 / kHpt retained rows of kHpt query heads of one KV group (row r of
+// the tile is head r / (128 / kHpt), entry r % (128 / kHpt)), and the CTA's second tile the next kHpt heads of that group.
+template <bool kSplit, int kHpt = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
-    static_assert(!(kSplit && kHeads), "the head-pair form is a variant of the shared form");
+    static_assert(!(kSplit && kHpt > 0), "the head forms are variants of the shared form");
+    static_assert(kHpt == 0 || kHpt == 1 || kHpt == 2, "one, two or four query heads per CTA");
     using C = Cfg<kSplit>;
-    // retained-list entries one CTA covers; kOneSpan: both softmax groups work on the SAME 128 entries (the split form:
-    // alternate K/V tiles; the head-pair form: two query heads of one KV group, so that the groups' K/V tile ranges and
+    constexpr bool kHeads = kHpt > 0;
+    // retained-list entries one CTA covers; kOneSpan: both softmax groups work on the SAME entries (the split form:
+    // alternate K/V tiles; the head forms: different query heads of one KV group, so that the groups' K/V tile ranges and
     // masks coincide and no tile is ever worked on by one group alone)
     constexpr bool kOneSpan = kSplit || kHeads;
-    constexpr int kRows = kOneSpan ? kTileM : C::kRows;
+    constexpr int kTileRows = kHeads ? kTileM / kHpt : kTileM;   // retained-list entries per Q tile
+    constexpr int kRows = kOneSpan ? kTileRows : C::kRows;
     constexpr int kStages = C::kStages, kOffQ = C::kOffQ, kOffRing = C::kOffRing, kOffBar = C::kOffBar, kStep = C::kStep;
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -248,7 +254,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     // instead of delaying the first wave of real work.  Any estimate gives a one-to-one assignment.
     int pair = p.first_pair - rb;
     if (pair < 0) pair += p.n_row_blocks;
-    constexpr int kHeadsPerCta = kHeads ? 2 : 1;
+    constexpr int kHeadsPerCta = kHeads ? 2 * kHpt : 1;
     const int qh = (bh % (p.Hq / kHeadsPerCta)) * kHeadsPerCta, b = bh / (p.Hq / kHeadsPerCta);   // first (or only) head
     const int nk = p.n_kept[b];
     const int slot0 = pair * kRows;
@@ -278,10 +284,10 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
 #pragma unroll
         for (int it = 0; it < kRounds; ++it) {
             const int rr = it * 16 + warp * 2 + (lane >> 4);           // row of the CTA's Q buffer (tile rr / 128)
-            const int s_q = slot0 + (kHeads ? (rr & (kTileM - 1)) : rr);
+            const int s_q = slot0 + (kHeads ? (rr & (kTileRows - 1)) : rr);
             tq[it] = s_q < nk ? kept[s_q] : -1;
         }
-        const int slot_pre = slot0 + (kOneSpan ? 0 : (warp >> 2) * kTileM) + (tid & (kTileM - 1));
+        const int slot_pre = slot0 + (kOneSpan ? 0 : (warp >> 2) * kTileM) + (tid & (kTileRows - 1));
         if (slot_pre < nk) t_row = kept[slot_pre];
     }
 
@@ -292,7 +298,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     for (int i = 0; i < kQTiles; ++i) {
         const int s_lo = slot0 + (kOneSpan ? 0 : i * kTileM);
         if (s_lo < nk) {
-            const int s_last = min(s_lo + kTileM, nk) - 1;
+            const int s_last = min(s_lo + kTileRows, nk) - 1;
             const int t_first = kept[s_lo], t_last = kept[s_last];
             int k_first = p.window > 0 ? max(0, t_first - p.window + 1) : 0;   // first key the tile's first row sees
             int k_last = t_last;                                                // last key its last row sees
@@ -432,7 +438,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         const int i = warp >> 2;                 // group: its Q tile (shared) or its half of the K/V tiles (split)
         const int r = tid & (kTileM - 1);        // row within the tile
-        const int slot = slot0 + (kOneSpan ? 0 : i * kTileM) + r;
+        const int slot = slot0 + (kOneSpan ? 0 : i * kTileM) + (r & (kTileRows - 1));
         const bool valid = slot < nk;               // t_row (fetched above) is the row's token position, -1 if none
         int hi = t_row;                                                           // visible keys: lo .. hi
         int lo = (valid && p.window > 0) ? max(0, t_row - p.window + 1) : 0;
@@ -446,8 +452,10 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             uint4 qv[kRounds];
             const __nv_bfloat16* qbase = p.Q + (long long)b * p.qs.b + (long long)qh * p.qs.h + cc * 8;
 #pragma unroll
-            for (int it = 0; it < kRounds; ++it)   // head-pair form: rounds 8..15 fill the second head's tile
-                qv[it] = tq[it] >= 0 ? ldg16(qbase + (kHeads ? (long long)(it >> 3) * p.qs.h : 0ll) + (long long)tq[it] * p.qs.t) : zero4;
+            for (int it = 0; it < kRounds; ++it) {   // head forms: rounds 8..15 fill the second tile, a round lies within one head
+                const int hh = kHeads ? (it >> 3) * kHpt + ((it & 7) * 16) / kTileRows : 0;
+                qv[it] = tq[it] >= 0 ? ldg16(qbase + (long long)hh * p.qs.h + (long long)tq[it] * p.qs.t) : zero4;
+            }
 #pragma unroll
             for (int it = 0; it < kRounds; ++it) {
                 const int rr = it * 16 + w8 * 2 + sub;
@@ -532,7 +540,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             __syncwarp();
             tc_fence_after();
             const float inv = 1.f / l_run;
-            __nv_bfloat16* Oi = Ob + (kHeads ? (long long)i * p.os.h : 0ll);   // this group's head
+            __nv_bfloat16* Oi = Ob + (kHeads ? (long long)(i * kHpt) * p.os.h : 0ll);   // this group's first head
             int* trow_s = reinterpret_cast<int*>(smem + kOffRing + 4096) + i * kTileM;
             trow_s[r] = t_row;
             uint8_t* stage = smem + kOffQ + i * kTileBytes + r * 256;
@@ -557,7 +565,7 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
             for (int pass = 0; pass < kTileM / 8; ++pass) {
                 const int R = pass * 8 + sub, t_out = trow_s[R];
                 if (t_out >= 0)
-                    *reinterpret_cast<uint4*>(Oi + (long long)t_out * p.os.t + l16 * 8) =
+                    *reinterpret_cast<uint4*>(Oi + (long long)(R / kTileRows) * p.os.h + (long long)t_out * p.os.t + l16 * 8) =
                         *reinterpret_cast<const uint4*>(smem + kOffQ + i * kTileBytes + R * 256 + ((l16 ^ (R & 15)) << 4));
             }
         }
@@ -889,7 +897,10 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg<false>::kSmemBytes);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attention_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(attention_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg<false>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attention_tc_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Cfg<false>::kSmemBytes);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -903,7 +914,8 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         // never answered by running another kernel.
         cudaFuncAttributes fa{};
         if (cudaFuncGetAttributes(&fa, attention_tc_kernel<false>) != cudaSuccess || fa.numRegs != 168 ||
-            cudaFuncGetAttributes(&fa, attention_tc_kernel<false, true>) != cudaSuccess || fa.numRegs != 168 ||
+            cudaFuncGetAttributes(&fa, attention_tc_kernel<false, 1>) != cudaSuccess || fa.numRegs != 168 ||
+            cudaFuncGetAttributes(&fa, attention_tc_kernel<false, 2>) != cudaSuccess || fa.numRegs != 168 ||
             cudaFuncGetAttributes(&fa, attention_tc_kernel<true>) != cudaSuccess || fa.numRegs != 168)
             return cudaErrorInvalidDeviceFunction;
         // the single form: 256 threads at 128 registers, traded 128 x 200 + 128 x 56
@@ -935,11 +947,15 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     const bool single = ctx->attention_form == 3;
     const bool split = ctx->attention_form == 2 || (ctx->attention_form == 0 && ctas_shared < 1.0 * sms);
     // Grouped-query attention with an even number of query heads per KV head: the two Q tiles of a shared-form CTA are
-    // the same 128 retained rows of two query heads of one group instead of 256 rows of one head.
-    const bool can_pair_heads = s.n_kv_heads > 0 && s.n_q_heads % s.n_kv_heads == 0 && (s.n_q_heads / s.n_kv_heads) % 2 == 0;
-    if (ctx->attention_form == 4 && !can_pair_heads) return cudaErrorNotSupported;
-    const bool heads = ctx->attention_form == 4 || (ctx->attention_form == 0 && !split && can_pair_heads);
-    const int rows_per_cta = (split || single || heads) ? kTileM : kQTiles * kTileM;
+    // the same 128 retained rows of two query heads of one group instead of 256 rows of one head; with a multiple of
+    // four, the same 64 rows of four heads (two per tile): the shorter the span of positions a CTA's rows cover, the
+    // fewer K/V tiles it has to visit beyond the window (or the causal triangle) itself.
+    const int q_per_kv = (s.n_kv_heads > 0 && s.n_q_heads % s.n_kv_heads == 0) ? s.n_q_heads / s.n_kv_heads : 1;
+    if ((ctx->attention_form == 4 && q_per_kv % 2) || (ctx->attention_form == 5 && q_per_kv % 4)) return cudaErrorNotSupported;
+    const int hpt = ctx->attention_form == 4 ? 1 : ctx->attention_form == 5 ? 2     // heads per Q tile, 0 = one head per CTA
+                  : (ctx->attention_form == 0 && !split) ? (q_per_kv % 4 == 0 ? 2 : q_per_kv % 2 == 0 ? 1 : 0) : 0;
+    const bool heads = hpt > 0;
+    const int rows_per_cta = heads ? kTileM / hpt : (split || single) ? kTileM : kQTiles * kTileM;
     tp.n_row_blocks = (s.seq + rows_per_cta - 1) / rows_per_cta;
     {
         const long long kept_est = (p.select_mode == TF_SELECT_RATIO) ? (long long)s.seq - (long long)floor(p.prune_ratio * (double)s.seq)
@@ -949,15 +965,16 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
     }
     const double kv_bytes = 2.0 * s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
     tp.heads_fastest = (kv_bytes <= 48e6 || ctas_shared < 6.0 * sms) ? 1 : 0;   // K and V stay in L2, or balance matters more
-    const long long n_ctas = (long long)tp.n_row_blocks * (heads ? s.n_q_heads / 2 : s.n_q_heads) * s.batch;
+    const long long n_ctas = (long long)tp.n_row_blocks * (heads ? s.n_q_heads / (2 * hpt) : s.n_q_heads) * s.batch;
     if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
     cudaError_t e;
     if (single) e = launch_dependent(attention_tc_single_kernel, dim3((unsigned)n_ctas), dim3(kThreads1), kSmemBytes1, st, tp, mapK, mapV);
-    else if (heads) e = launch_dependent(attention_tc_kernel<false, true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
+    else if (hpt == 2) e = launch_dependent(attention_tc_kernel<false, 2>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
+    else if (hpt == 1) e = launch_dependent(attention_tc_kernel<false, 1>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     else if (split) e = launch_dependent(attention_tc_kernel<true>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<true>::kSmemBytes, st, tp, mapK, mapV);
     else       e = launch_dependent(attention_tc_kernel<false>, dim3((unsigned)n_ctas), dim3(kThreads), Cfg<false>::kSmemBytes, st, tp, mapK, mapV);
     ctx->launches += 1;
-    ctx->last_attention_kernel = single ? TF_KERNEL_ATTN_TC_SINGLE : heads ? TF_KERNEL_ATTN_TC_HEAD_PAIR
+    ctx->last_attention_kernel = single ? TF_KERNEL_ATTN_TC_SINGLE : hpt == 2 ? TF_KERNEL_ATTN_TC_HEAD_QUAD : hpt == 1 ? TF_KERNEL_ATTN_TC_HEAD_PAIR
                                         : split ? TF_KERNEL_ATTN_TC_SPLIT : TF_KERNEL_ATTN_TC_SHARED;
     return e;
 }

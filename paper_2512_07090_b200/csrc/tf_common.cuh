@@ -173,7 +173,7 @@ struct tf_ctx {
     tf::ScanScratch scan_owned;    // ... and of owned_ws
     int use_tensor_cores;          // bf16 attention path
     int scan_path;                 // tf_kv_stats: 0 = choose, 1 = plain CUDA-core kernel, 2 / 3 = Gram-matrix kernel, one tile per CTA / persistent
-    int attention_form;            // tensor-core kernel: 0 = choose by shape and grid size, 1 = shared K/V tiles (two row tiles), 2 = split K/V tiles, 3 = single, 4 = shared K/V tiles (two query heads)
+    int attention_form;            // tensor-core kernel: 0 = choose by shape and grid size, 1 = shared K/V tiles (two row tiles), 2 = split K/V tiles, 3 = single, 4 / 5 = shared K/V tiles (two / four query heads of a KV group)
     long long launches;            // kernels launched through this context
     int last_scan_kernel;          // TF_KERNEL_* of the latest similarity scan / attention launched through this context
     int last_attention_kernel;

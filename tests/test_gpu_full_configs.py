@@ -72,7 +72,8 @@ def _check_layer(wl, layer, ratio, all_rows=False):
     assert code == tfb.TF_OK, det
     scan_kernel, attn_kernel = ctx.tf_last_kernels()
     assert scan_kernel in (tfb.TF_KERNEL_SCAN_GRAM_TILE, tfb.TF_KERNEL_SCAN_GRAM_PERSISTENT)
-    assert attn_kernel in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT, tfb.TF_KERNEL_ATTN_TC_HEAD_PAIR)
+    assert attn_kernel in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT, tfb.TF_KERNEL_ATTN_TC_HEAD_PAIR,
+                           tfb.TF_KERNEL_ATTN_TC_HEAD_QUAD)
 
     # ---- filter: in full against the oracle --------------------------------------------------------
     ref = oracle.select(ref_score, ratio, 4)

@@ -271,16 +271,16 @@ def test_select_few_candidates_left_with_ties_at_the_cut(S, n_tied):
 
 
 # ------------------------------------------------------------------------------- a5
-# path 2 / 3 / 4 / 5: the tensor-core kernel with K/V tiles shared by two Q tiles of one head / split between the softmax
-# groups / one Q tile and one softmax group per CTA, two CTAs per SM / shared by the same rows of two query heads of one
-# KV group (grouped-query shapes only)
+# path 2 / 3 / 4 / 5 / 6: the tensor-core kernel with K/V tiles shared by two Q tiles of one head / split between the softmax
+# groups / one Q tile and one softmax group per CTA, two CTAs per SM / shared by the same rows of two / four query heads of
+# one KV group (grouped-query shapes only)
 def _skip_unless_heads_pair(path, Hq, Hkv):
-    if path == 5 and (Hq // Hkv) % 2:
-        pytest.skip("the head-pair form needs an even number of query heads per KV head (its refusal has a test of its own)")
+    if path in (5, 6) and (Hq // Hkv) % {5: 2, 6: 4}[path]:
+        pytest.skip("the head forms need a multiple of two / four query heads per KV head (their refusal has a test of its own)")
 
 
 @pytest.mark.parametrize("dtype,tensor_cores", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 4), (torch.bfloat16, 5),
-                                                (torch.bfloat16, 1), (torch.bfloat16, 0), (torch.float32, 0)])
+                                                (torch.bfloat16, 6), (torch.bfloat16, 1), (torch.bfloat16, 0), (torch.float32, 0)])
 @pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5),
                                                     (1, 257, 8, 2, 0, 0.3), (2, 300, 4, 1, 64, 0.5),
                                                     (1, 515, 2, 2, 1, 0.7), (1, 200, 4, 2, 0, 0.99),
@@ -307,19 +307,20 @@ def test_pruned_attention_matches_oracle(dtype, tensor_cores, B, S, Hq, Hkv, win
 def _assert_attention_kernel(ctx, dtype, path):
     """The kernel that ran is the one the path names: 0 CUDA cores, 2 / 3 the tensor-core kernel's shared / split
     form (a build whose tensor-core kernel cannot be launched fails the call instead of running on CUDA cores),
-    4 / 5 its single and head-pair forms, 1 the tensor-core kernel in whichever form it chooses."""
+    4 / 5 / 6 its single, head-pair and head-quad forms, 1 the tensor-core kernel in whichever form it chooses."""
     ran = ctx.tf_last_kernels()[1]
     if dtype != torch.bfloat16 or path == 0:
         assert ran == tfb.TF_KERNEL_ATTN_SIMT
     elif path == 1:
-        assert ran in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT, tfb.TF_KERNEL_ATTN_TC_HEAD_PAIR)
+        assert ran in (tfb.TF_KERNEL_ATTN_TC_SHARED, tfb.TF_KERNEL_ATTN_TC_SPLIT, tfb.TF_KERNEL_ATTN_TC_HEAD_PAIR,
+                       tfb.TF_KERNEL_ATTN_TC_HEAD_QUAD)
     else:
         assert ran == {2: tfb.TF_KERNEL_ATTN_TC_SHARED, 3: tfb.TF_KERNEL_ATTN_TC_SPLIT, 4: tfb.TF_KERNEL_ATTN_TC_SINGLE,
-                       5: tfb.TF_KERNEL_ATTN_TC_HEAD_PAIR}[path]
+                       5: tfb.TF_KERNEL_ATTN_TC_HEAD_PAIR, 6: tfb.TF_KERNEL_ATTN_TC_HEAD_QUAD}[path]
 
 
 @pytest.mark.parametrize("dtype,path", [(torch.bfloat16, 2), (torch.bfloat16, 3), (torch.bfloat16, 4), (torch.bfloat16, 5),
-                                        (torch.bfloat16, 0), (torch.float32, 0)])
+                                        (torch.bfloat16, 6), (torch.bfloat16, 0), (torch.float32, 0)])
 @pytest.mark.parametrize("B,S,Hq,Hkv,window,ratio", [(1, 1, 2, 1, 0, 0.0), (2, 130, 4, 4, 0, 0.5), (1, 257, 8, 2, 0, 0.3),
                                                     (2, 300, 4, 1, 64, 0.5), (1, 515, 2, 2, 1, 0.7),
                                                     (1, 1300, 4, 2, 300, 0.5), (2, 1024, 2, 1, 0, 0.25)])
@@ -354,9 +355,9 @@ def test_layer_filter_retained_keys_only():
     assert n_mis == 0
 
 
-@pytest.mark.parametrize("path", [2, 3, 4, 5])
+@pytest.mark.parametrize("path", [2, 3, 4, 5, 6])
 def test_pruned_attention_nothing_kept_and_everything_kept(path):
-    q, k, v = _qkv(2, 70, 4 if path == 5 else 2, 2, torch.bfloat16)
+    q, k, v = _qkv(2, 70, {5: 4, 6: 8}.get(path, 2), 2, torch.bfloat16)
     g = Gpu(q, k, v)
     g.ctx.tf_set_attention_path(path)
     idx = torch.full((2, 70), -1, dtype=torch.int32, device=DEV)
@@ -371,12 +372,12 @@ def test_pruned_attention_nothing_kept_and_everything_kept(path):
     g.close()
 
 
-@pytest.mark.parametrize("tensor_cores", [2, 3, 4, 5])
+@pytest.mark.parametrize("tensor_cores", [2, 3, 4, 5, 6])
 @pytest.mark.parametrize("claimed_ratio", [0.0, 0.9])
 def test_pruned_attention_with_a_retained_list_the_ratio_does_not_predict(tensor_cores, claimed_ratio):
     """tf_pruned_attention takes any retained list; the kernel orders its row blocks by the count the prune ratio
     suggests.  With a list much longer or much shorter than that, every row block must still be served once."""
-    B, S, Hq, Hkv = 2, 1500, 4, 2
+    B, S, Hq, Hkv = 2, 1500, 8, 2
     q, k, v = _qkv(B, S, Hq, Hkv, torch.bfloat16, seed=5)
     qn, kn, vn = oracle_inputs(q, k, v)
     ref = oracle.layer_filter(qn, kn, vn, prune_ratio=0.4, warmup_tokens=1)      # the list really keeps 60 %
@@ -622,13 +623,14 @@ def test_requested_kernel_that_cannot_take_the_call_is_an_error_not_a_fallback()
             g.ctx.tf_kv_stats(g.shape, g.params, k, v, g.sim_k, g.sim_v)
         assert e.value.code == tfb.TF_ERR_UNSUPPORTED
     g.close()
-    q, k, v = _qkv(1, 200, 6, 2, torch.bfloat16)               # three query heads per KV head: no head pairs
-    g = Gpu(q, k, v)
-    g.ctx.tf_set_attention_path(5)
-    with pytest.raises(tfb.TokenFilterError) as e:
-        g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
-    assert e.value.code == tfb.TF_ERR_UNSUPPORTED
-    g.close()
+    for Hq, path in ((6, 5), (4, 6)):                          # three / two query heads per KV head: no pairs / no fours
+        q, k, v = _qkv(1, 200, Hq, 2, torch.bfloat16)
+        g = Gpu(q, k, v)
+        g.ctx.tf_set_attention_path(path)
+        with pytest.raises(tfb.TokenFilterError) as e:
+            g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
+        assert e.value.code == tfb.TF_ERR_UNSUPPORTED
+        g.close()
 
 
 # ------------------------------------------------------------------------------- online decode step
@@ -727,8 +729,8 @@ def test_layer_filter_random_shapes_modes_and_layouts(case):
     qn, kn, vn = oracle_inputs(q, k, v)
     ref = oracle.layer_filter(qn, kn, vn, window=window, **kw)
     g = Gpu(q, k, v, window=window, **kw)
-    path = int(rng.choice([1, 2, 3, 4, 5])) if dtype == torch.bfloat16 else 0
-    g.ctx.tf_set_attention_path(1 if path == 5 and (Hq // Hkv) % 2 else path)
+    path = int(rng.choice([1, 2, 3, 4, 5, 6])) if dtype == torch.bfloat16 else 0
+    g.ctx.tf_set_attention_path(1 if path in (5, 6) and (Hq // Hkv) % {5: 2, 6: 4}[path] else path)
     g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)
     g.status_ok()
     assert np.abs(to_np(g.score) - ref["score"]).max() < SCORE_ATOL
