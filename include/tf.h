@@ -163,6 +163,15 @@ tf_status tf_select(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *
                     const float *score, uint8_t *keep_mask, int32_t *kept_idx, int32_t *n_kept,
                     float *theta, void *stream);
 
+/* Steps a3 + a4 in one call (Alg. 1 from "(s_k, sigma_k^2)" to the skip decision; Eq. 2-3, Section 3.3): the
+ * arguments of tf_score_fuse followed by the outputs of tf_select, with the same meaning, layout and results (the
+ * scores have the bits tf_score_fuse gives, the selection the outputs tf_select gives on them).  For sequences of
+ * 4097 to 32768 tokens with up to 8 KV heads both steps run in one launch, a thread-block cluster per sequence;
+ * otherwise as two kernels.  theta may be NULL. */
+tf_status tf_score_select(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
+                          const float *sim_k, const float *sim_v, float *score, uint8_t *keep_mask,
+                          int32_t *kept_idx, int32_t *n_kept, float *theta, void *stream);
+
 /* Step a5 (Section 3.2: skipped tokens' attention output is zero; standard causal softmax
  * attention otherwise).  For every retained token kept_idx[b, i], i < n_kept[b], and query head
  * q: O = softmax(scale * Q.K^T over visible keys) V.  Every other row of O is set to zero, so O
@@ -270,6 +279,12 @@ tf_status tf_last_kernels(tf_ctx *ctx, int32_t kernels[2]);
  * kernel is a requirement:
  * a call it cannot take fails with TF_ERR_UNSUPPORTED instead of running another kernel.  For A/B checks. */
 tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
+
+/* Which kernel steps a3 / a4 use (tf_select, tf_score_select, tf_layer_filter): 0 = choose (default: a cluster of
+ * CTAs per sequence for 4097 to 32768 tokens, one CTA per sequence otherwise), 1 = one CTA per sequence (step a3 as
+ * a launch of its own), 2 = a cluster per sequence; a call whose sequence length it cannot take (up to 1024 or more
+ * than 32768 tokens) then fails with TF_ERR_UNSUPPORTED.  Same results either way.  For A/B checks. */
+tf_status tf_set_select_path(tf_ctx *ctx, int path);
 
 /* Which kernel tf_kv_stats uses: 0 = choose (default: by dtype, anchor mode and problem size), 1 = the
  * plain CUDA-core kernel (any dtype and anchor mode), 2 = the kernel that forms 128-token Gram matrices

@@ -32,7 +32,7 @@ EXPORTS = ("tf_default_params", "tf_create", "tf_destroy", "tf_workspace_bytes",
            "tf_kv_stats", "tf_kv_stats_static", "tf_score_fuse", "tf_select", "tf_pruned_attention", "tf_layer_filter",
            "tf_layer_filter_host", "tf_get_status", "tf_clear_status", "tf_set_attention_path",
            "tf_status_string", "tf_tail_policy", "tf_decode_step", "tf_set_scan_path", "tf_last_kernels",
-           "tf_set_wait_limits", "tf_wait_selftest")
+           "tf_set_wait_limits", "tf_wait_selftest", "tf_score_select", "tf_set_select_path")
 
 
 class tf_shape(C.Structure):
@@ -207,6 +207,10 @@ class Context:
         _check(lib().tf_select(self._h, C.byref(shape), C.byref(params), _ptr(score), _ptr(keep_mask),
                                _ptr(kept_idx), _ptr(n_kept), _ptr(theta), _stream()), "tf_select")
 
+    def tf_score_select(self, shape, params, sim_k, sim_v, score, keep_mask, kept_idx, n_kept, theta=None):
+        _check(lib().tf_score_select(self._h, C.byref(shape), C.byref(params), _ptr(sim_k), _ptr(sim_v), _ptr(score),
+                                     _ptr(keep_mask), _ptr(kept_idx), _ptr(n_kept), _ptr(theta), _stream()), "tf_score_select")
+
     def tf_pruned_attention(self, shape, params, Q, K, V, kept_idx, n_kept, O):
         _check(lib().tf_pruned_attention(self._h, C.byref(shape), C.byref(params), _ptr(Q), _ptr(K), _ptr(V),
                                          _ptr(kept_idx), _ptr(n_kept), _ptr(O), _stream()), "tf_pruned_attention")
@@ -240,8 +244,13 @@ class Context:
 
     def tf_set_attention_path(self, path):
         """0 / False: CUDA-core kernel; 1 / True: tensor-core kernel (form chosen by size); 2: shared form; 3: split form;
-        4: single form (one Q tile and one softmax group per CTA, two CTAs per SM)."""
+        4: single form (one Q tile and one softmax group per CTA, two CTAs per SM); 5 / 6: two / four query heads of one
+        KV group per CTA (grouped-query shapes)."""
         _check(lib().tf_set_attention_path(self._h, C.c_int(int(path))), "tf_set_attention_path")
+
+    def tf_set_select_path(self, path: int):
+        """0: choose; 1: selection by one CTA per sequence (fusion as its own launch); 2: fusion + selection by a cluster per sequence."""
+        _check(lib().tf_set_select_path(self._h, C.c_int(int(path))), "tf_set_select_path")
 
     def tf_set_scan_path(self, path: int):
         """0: choose; 1: plain CUDA-core similarity scan; 2: Gram-matrix scan on the tensor cores (bf16 sums), one tile per CTA; 3: the same, persistent."""

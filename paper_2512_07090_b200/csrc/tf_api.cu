@@ -236,7 +236,21 @@ tf_status tf_select(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* 
     if (!g.ok) return TF_ERR_CUDA;
     cudaError_t e = launch_select(ctx, *shape, *params, score, keep_mask, kept_idx, n_kept, theta,
                                   static_cast<cudaStream_t>(stream));
-    return e == cudaSuccess ? TF_OK : TF_ERR_CUDA;
+    return to_status(e);
+}
+
+tf_status tf_score_select(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params,
+                          const float* sim_k, const float* sim_v, float* score, uint8_t* keep_mask,
+                          int32_t* kept_idx, int32_t* n_kept, float* theta, void* stream) {
+    if (!ctx) return TF_ERR_INVALID_ARG;
+    tf_status s = check_shape(shape);
+    if (s == TF_OK) s = check_params(params);
+    if (s != TF_OK) return s;
+    if (!sim_k || !sim_v || !score || !keep_mask || !kept_idx || !n_kept) return TF_ERR_INVALID_ARG;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return TF_ERR_CUDA;
+    return to_status(launch_score_select(ctx, *shape, *params, sim_k, sim_v, score, keep_mask, kept_idx, n_kept, theta,
+                                         static_cast<cudaStream_t>(stream)));
 }
 
 tf_status tf_pruned_attention(tf_ctx* ctx, const tf_shape* shape, const tf_filter_params* params,
@@ -286,8 +300,7 @@ tf_status tf_layer_filter(tf_ctx* ctx, const tf_shape* shape, const tf_filter_pa
 
     ScanScratch* scan = (ctx->workspace == ctx->owned_ws && ctx->owned_ws) ? &ctx->scan_owned : &ctx->scan_user;
     cudaError_t e = launch_kv_stats(ctx, *shape, *params, K, V, sim_k, sim_v, nullptr, scan, st);
-    if (e == cudaSuccess) e = launch_score_fuse(ctx, *shape, *params, sim_k, sim_v, score, st);
-    if (e == cudaSuccess) e = launch_select(ctx, *shape, *params, score, keep_mask, kept_idx, n_kept, theta, st);
+    if (e == cudaSuccess) e = launch_score_select(ctx, *shape, *params, sim_k, sim_v, score, keep_mask, kept_idx, n_kept, theta, st);
     if (e != cudaSuccess) return to_status(e);
     void* kv_compact = nullptr;
     s = kv_compact_section(ctx, *shape, *params, &kv_compact);
@@ -380,8 +393,7 @@ tf_status tf_layer_filter_host(tf_ctx* ctx, const tf_shape* shape, const tf_filt
         float* theta = reinterpret_cast<float*>(ws + w.theta);
         tf_shape ds = *shape;                                  // device copies are dense like the host tensors
         e = launch_kv_stats(ctx, ds, *params, dK, dV, sim_k, sim_v, nullptr, &ctx->scan_owned, st);
-        if (e == cudaSuccess) e = launch_score_fuse(ctx, ds, *params, sim_k, sim_v, dS, st);
-        if (e == cudaSuccess) e = launch_select(ctx, ds, *params, dS, dM, dI, dN, theta, st);
+        if (e == cudaSuccess) e = launch_score_select(ctx, ds, *params, sim_k, sim_v, dS, dM, dI, dN, theta, st);
         if (e == cudaSuccess) e = cudaEventRecord(ev_sel, st);
     }
     s = to_status(e);
@@ -504,6 +516,12 @@ tf_status tf_set_attention_path(tf_ctx* ctx, int use_tensor_cores) {
     if (use_tensor_cores < 0 || use_tensor_cores > 6) return TF_ERR_INVALID_ARG;
     ctx->use_tensor_cores = use_tensor_cores ? 1 : 0;
     ctx->attention_form = use_tensor_cores >= 2 ? use_tensor_cores - 1 : 0;
+    return TF_OK;
+}
+
+tf_status tf_set_select_path(tf_ctx* ctx, int path) {
+    if (!ctx || path < 0 || path > 2) return TF_ERR_INVALID_ARG;
+    ctx->select_form = path;
     return TF_OK;
 }
 

@@ -84,22 +84,35 @@ __device__ __forceinline__ int first_kept_at_or_after(const int32_t* kept, int n
 // ---- step a3: mean / population variance over heads, weight alpha (Eq. 2, either reading), fused score (Eq. 3) ----
 __device__ __forceinline__ float fuse_alpha(int mode, float var_k, float var_v, float eps) {
     switch (mode) {
-        case TF_FUSE_EQ2_LITERAL: return (var_k + eps) / (var_k + var_v + 2.f * eps);
+        case TF_FUSE_EQ2_LITERAL: return __fdiv_rn(__fadd_rn(var_k, eps), __fmaf_rn(2.f, eps, __fadd_rn(var_k, var_v)));
         case TF_FUSE_KEY_ONLY: return 1.f;
         case TF_FUSE_VALUE_ONLY: return 0.f;
         case TF_FUSE_MEAN: return 0.5f;
-        default: return (var_v + eps) / (var_k + var_v + 2.f * eps);
+        default: return __fdiv_rn(__fadd_rn(var_v, eps), __fmaf_rn(2.f, eps, __fadd_rn(var_k, var_v)));
     }
 }
 __device__ __forceinline__ float fuse_score(int mode, float mean_k, float var_k, float mean_v, float var_v, float eps) {
+    // every rounding is spelled out: the kernels that evaluate this (one launch for step a3 alone, one for a3 + a4)
+    // must give the same bits whatever the compiler would contract
     const float alpha = fuse_alpha(mode, var_k, var_v, eps);
-    return (alpha * mean_k + (1.f - alpha) * mean_v) + 0.f;   // -0 -> +0
+    return __fadd_rn(__fmaf_rn(alpha, mean_k, __fmul_rn(__fsub_rn(1.f, alpha), mean_v)), 0.f);   // -0 -> +0
 }
 __device__ __forceinline__ void note_nan_score(DevStatus* st, float s, unsigned long long token) {
     if (s != s && st) {
         atomicAdd(&st->nan_count, 1ull);
         report_error(st, TF_ERR_NAN_SCORE, token);
     }
+}
+
+// ---- step a4: monotone map float -> uint32 (larger score <=> larger key); -0 and +0 share a key ----
+__device__ __forceinline__ unsigned int score_key(float s) {
+    if (s == 0.f) s = 0.f;
+    const unsigned int u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_score(unsigned int k) {
+    const unsigned int u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+    return __uint_as_float(u);
 }
 
 // ---- host-side launch bookkeeping --------------------------------------------------------------
@@ -173,6 +186,7 @@ struct tf_ctx {
     tf::ScanScratch scan_owned;    // ... and of owned_ws
     int use_tensor_cores;          // bf16 attention path
     int scan_path;                 // tf_kv_stats: 0 = choose, 1 = plain CUDA-core kernel, 2 / 3 = Gram-matrix kernel, one tile per CTA / persistent
+    int select_form;               // selection: 0 = choose by sequence length, 1 = one CTA per sequence, 2 = a cluster per sequence
     int attention_form;            // tensor-core kernel: 0 = choose by shape and grid size, 1 = shared K/V tiles (two row tiles), 2 = split K/V tiles, 3 = single, 4 / 5 = shared K/V tiles (two / four query heads of a KV group)
     long long launches;            // kernels launched through this context
     int last_scan_kernel;          // TF_KERNEL_* of the latest similarity scan / attention launched through this context
@@ -229,6 +243,17 @@ cudaError_t launch_score_fuse(tf_ctx* ctx, const tf_shape& s, const tf_filter_pa
 cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                           const float* score, uint8_t* keep_mask, int32_t* kept_idx,
                           int32_t* n_kept, float* theta, cudaStream_t st);
+// steps a3 + a4 by a thread-block cluster per sequence (tf_select_cluster.cu); sim_k == nullptr: a4 alone on `score`
+bool select_cluster_usable(const tf_shape& s);      // sequence lengths it can take
+bool select_cluster_preferred(const tf_shape& s);   // ... and those it is chosen for
+bool select_cluster_fuses(const tf_shape& s);       // step a3 inside the same launch (up to 8 KV heads)
+cudaError_t launch_select_cluster(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const float* sim_k,
+                                  const float* sim_v, float* score, uint8_t* keep_mask, int32_t* kept_idx,
+                                  int32_t* n_kept, float* theta, cudaStream_t st);
+// a3 then a4: one launch where the cluster form takes the sequence length, else the two kernels
+cudaError_t launch_score_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const float* sim_k,
+                                const float* sim_v, float* score, uint8_t* keep_mask, int32_t* kept_idx,
+                                int32_t* n_kept, float* theta, cudaStream_t st);
 cudaError_t launch_attention_simt(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p,
                                   const void* Q, const void* K, const void* V,
                                   const int32_t* kept_idx, const int32_t* n_kept, void* O,

@@ -21,17 +21,6 @@ constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kMaxTableChunks = 64;   // longer sequences (> 65536 tokens) fall back to two block scans per 1024 tokens
 
-// Monotone map float -> uint32 (larger score <=> larger key); -0 and +0 share a key.
-__device__ __forceinline__ unsigned int score_key(float s) {
-    if (s == 0.f) s = 0.f;
-    const unsigned int u = __float_as_uint(s);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float key_score(unsigned int k) {
-    const unsigned int u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
-    return __uint_as_float(u);
-}
-
 struct SelectParams {
     const float* score;        // [B,S]
     const uint8_t* eligible;   // [B,S] or null
@@ -456,6 +445,9 @@ cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params
                           const float* score, uint8_t* keep_mask, int32_t* kept_idx,
                           int32_t* n_kept, float* theta, cudaStream_t st) {
     if (s.batch == 0) return cudaSuccess;
+    // long sequences (4097 to 32768 tokens) are shared by the CTAs of a cluster
+    if (ctx->select_form == 2 || (ctx->select_form == 0 && select_cluster_preferred(s)))
+        return launch_select_cluster(ctx, s, p, nullptr, nullptr, const_cast<float*>(score), keep_mask, kept_idx, n_kept, theta, st);
     SelectParams sp{};
     sp.score = score; sp.eligible = p.eligible; sp.threshold = p.threshold;
     sp.S = s.seq; sp.warmup = p.warmup_tokens; sp.mode = p.select_mode;
@@ -463,6 +455,17 @@ cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params
     sp.keep_mask = keep_mask; sp.kept_idx = kept_idx; sp.n_kept = n_kept; sp.theta = theta;
     cudaError_t e = launch_select_form(sp, s.batch, st);
     ctx->launches += 1;
+    return e;
+}
+
+cudaError_t launch_score_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params& p, const float* sim_k,
+                                const float* sim_v, float* score, uint8_t* keep_mask, int32_t* kept_idx,
+                                int32_t* n_kept, float* theta, cudaStream_t st) {
+    if ((ctx->select_form == 2 && select_cluster_usable(s) && select_cluster_fuses(s)) ||
+        (ctx->select_form == 0 && select_cluster_preferred(s) && select_cluster_fuses(s)))
+        return launch_select_cluster(ctx, s, p, sim_k, sim_v, score, keep_mask, kept_idx, n_kept, theta, st);
+    cudaError_t e = launch_score_fuse(ctx, s, p, sim_k, sim_v, score, st);
+    if (e == cudaSuccess) e = launch_select(ctx, s, p, score, keep_mask, kept_idx, n_kept, theta, st);
     return e;
 }
 

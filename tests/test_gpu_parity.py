@@ -213,15 +213,74 @@ def _select_case(score, ratio, warm, elig=None, mode=tfb.TF_SELECT_RATIO, thr=No
     if thr is not None:
         th_t = torch.from_numpy(np.asarray(thr, np.float32)).to(DEV); kw["threshold"] = th_t
     g = Gpu(q, q, q, **kw)
-    g.ctx.tf_select(g.shape, g.params, sc, g.keep, g.idx, g.nk, g.theta)
-    g.status_ok()
     thr64 = None if thr is None else np.asarray(thr, np.float32).astype(np.float64)   # the same fp32 values
     ref = oracle.select(score.astype(np.float64), ratio, warm, elig, mode, thr64)
-    assert np.array_equal(g.keep.cpu().numpy(), ref["keep_mask"])
-    assert np.array_equal(g.idx.cpu().numpy(), ref["kept_idx"])
-    assert np.array_equal(g.nk.cpu().numpy(), ref["n_kept"])
-    assert np.array_equal(g.theta.cpu().numpy().astype(np.float64), ref["theta"])
+    # path 1: one CTA per sequence; path 2: a cluster of CTAs per sequence (1025 to 32768 tokens); 0: the library's choice
+    for path in ([0, 1, 2] if CLUSTER_SELECT_MIN < S <= CLUSTER_SELECT_MAX else [0, 1]):
+        g.ctx.tf_set_select_path(path)
+        for t in (g.keep, g.idx, g.nk):
+            t.fill_(77)
+        g.theta.fill_(float("nan"))
+        g.ctx.tf_select(g.shape, g.params, sc, g.keep, g.idx, g.nk, g.theta)
+        g.status_ok()
+        assert np.array_equal(g.keep.cpu().numpy(), ref["keep_mask"]), path
+        assert np.array_equal(g.idx.cpu().numpy(), ref["kept_idx"]), path
+        assert np.array_equal(g.nk.cpu().numpy(), ref["n_kept"]), path
+        assert np.array_equal(g.theta.cpu().numpy().astype(np.float64), ref["theta"]), path
     g.close()
+
+
+CLUSTER_SELECT_MIN, CLUSTER_SELECT_MAX = 1024, 32768   # sequence lengths the cluster form of steps a3 + a4 takes
+
+
+@pytest.mark.parametrize("S", [1025, 1500, 2048, 2049, 4096, 5000, 16384, 20000, 32768])
+@pytest.mark.parametrize("H,mode", [(1, tfb.TF_FUSE_INVVAR), (2, tfb.TF_FUSE_EQ2_LITERAL), (8, tfb.TF_FUSE_INVVAR),
+                                    (8, tfb.TF_FUSE_KEY_ONLY), (12, tfb.TF_FUSE_VALUE_ONLY), (32, tfb.TF_FUSE_MEAN),
+                                    (40, tfb.TF_FUSE_INVVAR)])
+def test_score_select_in_one_launch_gives_the_bits_of_the_two_steps(S, H, mode):
+    """tf_score_select (steps a3 + a4, a cluster per sequence) against tf_score_fuse followed by tf_select with one CTA
+    per sequence: the same score bits, the same masks, lists, counts and thresholds; and both against the oracle."""
+    B = 3
+    rng = np.random.default_rng(S + H)
+    ck = rng.uniform(-0.3, 0.9, (B, S, H)).astype(np.float32)
+    cv = rng.uniform(-0.3, 0.9, (B, S, H)).astype(np.float32)
+    ck[0, 5] = 0.25; cv[0, 5] = -0.5                       # zero variance on both sides
+    ck[1, 700:720] = ck[1, 699]; cv[1, 700:720] = cv[1, 699]   # exactly equal scores
+    q, k, v = _qkv(B, S, H, H, torch.bfloat16)
+    g = Gpu(q, k, v, fuse_mode=mode, prune_ratio=0.5, warmup_tokens=4)
+    ck_d, cv_d = torch.from_numpy(ck).to(DEV), torch.from_numpy(cv).to(DEV)
+    g.ctx.tf_set_select_path(1)
+    g.ctx.tf_score_fuse(g.shape, g.params, ck_d, cv_d, g.score)
+    g.ctx.tf_select(g.shape, g.params, g.score, g.keep, g.idx, g.nk, g.theta)
+    g.status_ok()
+    two = [t.clone() for t in (g.score, g.keep, g.idx, g.nk, g.theta)]
+    for path in (2, 0):
+        g.ctx.tf_set_select_path(path)
+        g.score.fill_(float("nan")); g.keep.fill_(77); g.idx.fill_(77); g.nk.fill_(77); g.theta.fill_(float("nan"))
+        launches = g.ctx.tf_get_status()[1]["launches"]
+        g.ctx.tf_score_select(g.shape, g.params, ck_d, cv_d, g.score, g.keep, g.idx, g.nk, g.theta)
+        g.status_ok()
+        one_launch = H <= 8 and (path == 2 or S > 4096)     # step a3 joins the cluster's launch for up to 8 KV heads
+        assert g.ctx.tf_get_status()[1]["launches"] == launches + (1 if one_launch else 2)
+        for got, want in zip((g.score, g.keep, g.idx, g.nk, g.theta), two):
+            assert torch.equal(got.view(torch.int32) if got.dtype == torch.float32 else got,
+                               want.view(torch.int32) if want.dtype == torch.float32 else want), path
+    score = to_np(g.score)
+    assert np.abs(score - oracle.score_fuse(ck, cv, mode)).max() < 2e-6
+    ref = oracle.select(score, 0.5, 4)
+    assert np.array_equal(g.keep.cpu().numpy(), ref["keep_mask"]) and np.array_equal(g.idx.cpu().numpy(), ref["kept_idx"])
+    g.close()
+
+
+def test_cluster_selection_refuses_lengths_it_cannot_take():
+    for S in (1000, 40000):
+        q = torch.zeros(1, S, 1, 128, dtype=torch.bfloat16, device=DEV)
+        g = Gpu(q, q, q)
+        g.ctx.tf_set_select_path(2)
+        with pytest.raises(tfb.TokenFilterError) as e:
+            g.ctx.tf_select(g.shape, g.params, g.score, g.keep, g.idx, g.nk, g.theta)
+        assert e.value.code == tfb.TF_ERR_UNSUPPORTED
+        g.close()
 
 
 @pytest.mark.parametrize("S", [1, 2, 31, 1024, 1025, 2048, 2049, 5000, 8193, 16384, 16385, 40000, 51200, 60000, 70000])   # register forms of 2, 4, 8, 16 scores per thread, then scores staged in shared memory (up to 51200), then re-read from global memory (one-scan sweep up to 65536 tokens, block scans beyond)
