@@ -808,13 +808,14 @@ def test_layer_filter_replayed_from_a_cuda_graph_with_new_inputs():
     """One tf_layer_filter call captured into a CUDA graph (after a first call outside the capture, which clears the
     scratch and sets function attributes) and replayed over buffers whose contents change between replays: everything a
     launch needs to tell its own look-back records from an earlier launch's lives on the device, so every replay is
-    right.  Both Gram-scan kernels and the CUDA-core scan."""
+    right.  Both Gram-scan kernels and the CUDA-core scan; fusion and selection as two launches and as the cluster launch."""
     B, S, Hq, Hkv = 2, 1300, 8, 2
     inputs = [_qkv(B, S, Hq, Hkv, torch.bfloat16, seed=90 + i) for i in range(3)]
-    for scan_path in (2, 3, 1):
+    for scan_path, select_path in ((2, 1), (3, 2), (1, 2)):
         q, k, v = (t.clone() for t in inputs[0])
         g = Gpu(q, k, v, prune_ratio=0.5, warmup_tokens=4)
         g.ctx.tf_set_scan_path(scan_path)
+        g.ctx.tf_set_select_path(select_path)
         g.ctx.tf_layer_filter(g.shape, g.params, q, k, v, g.O, g.score, g.keep, g.idx, g.nk)     # outside the capture
         torch.cuda.synchronize()
         side = torch.cuda.Stream()
