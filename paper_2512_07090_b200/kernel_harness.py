@@ -2,10 +2,11 @@
 program a profiler capture wants (a few hundred MB on the device instead of a whole workload ring).
 
     python -m paper_2512_07090_b200.kernel_harness --stage scan --batch 8 --seq 16384 --kv-heads 8 [--q-heads 32]
-           [--window 4096] [--prune 0.5] [--anchor ema --gamma 0.9] [--launches 6] [--scan-path 0..3] [--attention-path 0..4]
+           [--window 4096] [--prune 0.5] [--anchor ema --gamma 0.9] [--launches 6] [--scan-path 0..3] [--attention-path 0..6]
+           [--select-path 0..2]
 
-Stages: scan (tf_kv_stats), fuse (tf_score_fuse), select (tf_select), attention (tf_pruned_attention), step
-(tf_layer_filter).  Inputs are N(0,1) bf16 tensors from a fixed seed with a quarter of the tokens near-duplicates of an
+Stages: scan (tf_kv_stats), fuse (tf_score_fuse), select (tf_select), score_select (tf_score_select), attention
+(tf_pruned_attention), step (tf_layer_filter).  Inputs are N(0,1) bf16 tensors from a fixed seed with a quarter of the tokens near-duplicates of an
 earlier token (the recipe of the reduced parity cases); the stages before the requested one run once to produce its
 inputs.  Prints the mean time per launch from CUDA events.
 """
@@ -20,7 +21,7 @@ from . import binding as tfb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--stage", default="scan", choices=["scan", "fuse", "select", "attention", "step"])
+    ap.add_argument("--stage", default="scan", choices=["scan", "fuse", "select", "score_select", "attention", "step"])
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--seq", type=int, default=16384)
     ap.add_argument("--kv-heads", type=int, default=8)
@@ -32,6 +33,7 @@ def main():
     ap.add_argument("--launches", type=int, default=6)
     ap.add_argument("--scan-path", type=int, default=0)
     ap.add_argument("--attention-path", type=int, default=1)
+    ap.add_argument("--select-path", type=int, default=0)
     a = ap.parse_args()
     dev = "cuda:0"
     torch.cuda.set_device(0)
@@ -57,6 +59,7 @@ def main():
     ctx.ensure_workspace(shape, params)
     ctx.tf_set_scan_path(a.scan_path)
     ctx.tf_set_attention_path(a.attention_path)
+    ctx.tf_set_select_path(a.select_path)
     sim_k = torch.empty(B, S, Hkv, device=dev); sim_v = torch.empty_like(sim_k)
     score = torch.empty(B, S, device=dev)
     keep = torch.empty(B, S, dtype=torch.uint8, device=dev)
@@ -71,6 +74,7 @@ def main():
         if a.stage == "scan": ctx.tf_kv_stats(shape, params, k, v, sim_k, sim_v)
         elif a.stage == "fuse": ctx.tf_score_fuse(shape, params, sim_k, sim_v, score)
         elif a.stage == "select": ctx.tf_select(shape, params, score, keep, idx, nk)
+        elif a.stage == "score_select": ctx.tf_score_select(shape, params, sim_k, sim_v, score, keep, idx, nk)
         elif a.stage == "attention": ctx.tf_pruned_attention(shape, params, q, k, v, idx, nk, O)
         else: ctx.tf_layer_filter(shape, params, q, k, v, O, score, keep, idx, nk)
 
