@@ -39,6 +39,7 @@ struct ClusterSelectParams {
     const float* threshold;                   // [B] (threshold mode)
     int S, H, warmup, mode, fuse_mode;
     float eps;
+    int vec4;                                 // the similarities can be read as float4 (H a multiple of 4, 16-byte aligned)
     long long p_target;                       // floor(ratio*S), computed on the host in double
     uint8_t* keep_mask; int32_t* kept_idx; int32_t* n_kept; float* theta;
     DevStatus* status;
@@ -83,6 +84,8 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Clu
     __shared__ unsigned int s_prefix;
     __shared__ int s_rank, s_count, s_total;
     __shared__ int s_tab[KPT * kCsWarps];     // [chunk][warp] ballot counts of the final sweep
+    __shared__ unsigned int s_few[32];        // CTA 0's copy: the last few candidates' keys, appended by the whole cluster
+    __shared__ int s_few_n;
 
     grid_launch_dependents();   // few CTAs: the attention grid may take the other SMs and set up meanwhile
     grid_dependency_wait();
@@ -93,6 +96,7 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Clu
     const int t_base = rank * (KPT * kCsThreads);
     const uint8_t* el = p.eligible ? p.eligible + (size_t)b * S : nullptr;
     float* sc = p.score + (size_t)b * S;
+    if (tid == 0) s_few_n = 0;                // used at most once, after at least one cluster barrier
 
     // token of slot i: t_base + i*512 + tid (ascending in (i, tid))
     float sreg[KPT];
@@ -107,10 +111,23 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Clu
             for (int u = 0; u < kBatch; ++u) {
                 const int t = t_base + (i0 + u) * kCsThreads + tid;
                 const size_t row = ((size_t)b * S + (t < S ? t : 0)) * p.H;
+                if (p.vec4) {
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    xk[u][h] = (t < S && h < p.H) ? __ldg(p.sim_k + row + h) : 0.f;
-                    xv[u][h] = (t < S && h < p.H) ? __ldg(p.sim_v + row + h) : 0.f;
+                    for (int h4 = 0; h4 < 2; ++h4) {
+                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), c = a;
+                        if (t < S && h4 * 4 < p.H) {
+                            a = __ldg(reinterpret_cast<const float4*>(p.sim_k + row) + h4);
+                            c = __ldg(reinterpret_cast<const float4*>(p.sim_v + row) + h4);
+                        }
+                        xk[u][4 * h4] = a.x; xk[u][4 * h4 + 1] = a.y; xk[u][4 * h4 + 2] = a.z; xk[u][4 * h4 + 3] = a.w;
+                        xv[u][4 * h4] = c.x; xv[u][4 * h4 + 1] = c.y; xv[u][4 * h4 + 2] = c.z; xv[u][4 * h4 + 3] = c.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int h = 0; h < 8; ++h) {
+                        xk[u][h] = (t < S && h < p.H) ? __ldg(p.sim_k + row + h) : 0.f;
+                        xv[u][h] = (t < S && h < p.H) ? __ldg(p.sim_v + row + h) : 0.f;
+                    }
                 }
             }
 #pragma unroll
@@ -204,6 +221,41 @@ __global__ void __launch_bounds__(kCsThreads, 1) select_cluster_kernel(const Clu
             n_eq = s_count;
             mask |= 255u << shift;
             __syncthreads();     // s_warp, s_prefix, s_rank and s_count are written again in the next pass
+            // Few candidates left under this prefix (typical after two or three passes): they are collected in CTA 0's
+            // shared memory and every CTA ranks them there instead of further histogram passes.  Same result: the key of
+            // rank r among them, how many candidates carry it, and the rank within those.  (n_eq is the same in every CTA.)
+            if (shift > 0 && n_eq <= 32) {
+                unsigned int* few0 = cluster.map_shared_rank(s_few, 0);
+                int* few_n0 = cluster.map_shared_rank(&s_few_n, 0);
+#pragma unroll
+                for (int i = 0; i < KPT; ++i) {
+                    const int t = t_base + i * kCsThreads + tid;
+                    if (t < S && candidate(t, sreg[i])) {
+                        const unsigned int k = score_key(sreg[i]);
+                        if ((k & mask) == prefix) few0[atomicAdd(few_n0, 1)] = k;     // exactly n_eq appends in all
+                    }
+                }
+                cluster.sync();
+                if (tid < 32) {
+                    const unsigned int key = tid < n_eq ? few0[tid] : 0u;
+                    int greater = 0, equal = 0;
+                    for (int o = 0; o < n_eq; ++o) {
+                        const unsigned int ko = __shfl_sync(0xffffffffu, key, o);
+                        greater += ko > key ? 1 : 0;
+                        equal += ko == key ? 1 : 0;
+                    }
+                    if (tid < n_eq && greater < r && r <= greater + equal) {   // every lane holding that key writes the same
+                        s_prefix = key;
+                        s_rank = r - greater;
+                        s_count = equal;
+                    }
+                }
+                __syncthreads();
+                prefix = s_prefix;
+                r = s_rank;
+                n_eq = s_count;
+                break;
+            }
         }
         key_thr = prefix;
         take_eq = r;             // 1 <= r <= n_eq
@@ -357,6 +409,7 @@ cudaError_t launch_select_cluster(tf_ctx* ctx, const tf_shape& s, const tf_filte
     cp.eligible = p.eligible; cp.threshold = p.threshold;
     cp.S = s.seq; cp.H = s.n_kv_heads; cp.warmup = p.warmup_tokens; cp.mode = p.select_mode; cp.fuse_mode = p.fuse_mode;
     cp.eps = p.var_eps > 0.f ? p.var_eps : 1e-8f;
+    cp.vec4 = (sim_k && s.n_kv_heads % 4 == 0 && ((reinterpret_cast<uintptr_t>(sim_k) | reinterpret_cast<uintptr_t>(sim_v)) & 15) == 0) ? 1 : 0;
     cp.p_target = (long long)floor(p.prune_ratio * (double)s.seq);
     cp.keep_mask = keep_mask; cp.kept_idx = kept_idx; cp.n_kept = n_kept; cp.theta = theta;
     cp.status = ctx->dev_status;
