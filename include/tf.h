@@ -166,7 +166,7 @@ tf_status tf_select(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *
 /* Steps a3 + a4 in one call (Alg. 1 from "(s_k, sigma_k^2)" to the skip decision; Eq. 2-3, Section 3.3): the
  * arguments of tf_score_fuse followed by the outputs of tf_select, with the same meaning, layout and results (the
  * scores have the bits tf_score_fuse gives, the selection the outputs tf_select gives on them).  For sequences of
- * 4097 to 32768 tokens with up to 8 KV heads both steps run in one launch, a thread-block cluster per sequence;
+ * 1025 to 32768 tokens with up to 8 KV heads both steps run in one launch, a thread-block cluster per sequence;
  * otherwise as two kernels.  theta may be NULL. */
 tf_status tf_score_select(tf_ctx *ctx, const tf_shape *shape, const tf_filter_params *params,
                           const float *sim_k, const float *sim_v, float *score, uint8_t *keep_mask,
@@ -281,7 +281,7 @@ tf_status tf_last_kernels(tf_ctx *ctx, int32_t kernels[2]);
 tf_status tf_set_attention_path(tf_ctx *ctx, int use_tensor_cores);
 
 /* Which kernel steps a3 / a4 use (tf_select, tf_score_select, tf_layer_filter): 0 = choose (default: a cluster of
- * CTAs per sequence for 4097 to 32768 tokens, one CTA per sequence otherwise), 1 = one CTA per sequence (step a3 as
+ * CTAs per sequence for 1025 to 32768 tokens, one CTA per sequence otherwise), 1 = one CTA per sequence (step a3 as
  * a launch of its own), 2 = a cluster per sequence; a call whose sequence length it cannot take (up to 1024 or more
  * than 32768 tokens) then fails with TF_ERR_UNSUPPORTED.  Same results either way.  For A/B checks. */
 tf_status tf_set_select_path(tf_ctx *ctx, int path);

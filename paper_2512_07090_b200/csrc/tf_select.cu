@@ -445,7 +445,7 @@ cudaError_t launch_select(tf_ctx* ctx, const tf_shape& s, const tf_filter_params
                           const float* score, uint8_t* keep_mask, int32_t* kept_idx,
                           int32_t* n_kept, float* theta, cudaStream_t st) {
     if (s.batch == 0) return cudaSuccess;
-    // long sequences (4097 to 32768 tokens) are shared by the CTAs of a cluster
+    // sequences of 1025 to 32768 tokens are shared by the CTAs of a cluster
     if (ctx->select_form == 2 || (ctx->select_form == 0 && select_cluster_preferred(s)))
         return launch_select_cluster(ctx, s, p, nullptr, nullptr, const_cast<float*>(score), keep_mask, kept_idx, n_kept, theta, st);
     SelectParams sp{};

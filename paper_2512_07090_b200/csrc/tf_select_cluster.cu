@@ -391,11 +391,11 @@ cudaError_t launch_form(const ClusterSelectParams& cp, int batch, int n_ranks, c
 
 }  // namespace
 
-// Sequence lengths the cluster form takes: more than 1024 tokens and at most 8 CTAs x 512 threads x 8 scores per
-// thread.  It is preferred from 4097 tokens on: up to there one CTA per sequence is as fast (the cluster's barriers
-// and remote histogram reads cost what the shorter passes save).
+// Sequence lengths the cluster form takes, and is chosen for: more than 1024 tokens (up to there one CTA per sequence
+// is as fast: the cluster's barriers and remote reads cost what the shorter passes save) and at most 8 CTAs x 512
+// threads x 8 scores per thread.
 bool select_cluster_usable(const tf_shape& s) { return s.seq > 1024 && s.seq <= 8 * kCsThreads * 8; }
-bool select_cluster_preferred(const tf_shape& s) { return s.seq > 4096 && select_cluster_usable(s); }
+bool select_cluster_preferred(const tf_shape& s) { return select_cluster_usable(s); }
 bool select_cluster_fuses(const tf_shape& s) { return s.n_kv_heads <= kFuseLanes; }
 
 // sim_k == nullptr: selection only, the scores are read from `score`

@@ -260,7 +260,7 @@ def test_score_select_in_one_launch_gives_the_bits_of_the_two_steps(S, H, mode):
         launches = g.ctx.tf_get_status()[1]["launches"]
         g.ctx.tf_score_select(g.shape, g.params, ck_d, cv_d, g.score, g.keep, g.idx, g.nk, g.theta)
         g.status_ok()
-        one_launch = H <= 8 and (path == 2 or S > 4096)     # step a3 joins the cluster's launch for up to 8 KV heads
+        one_launch = H <= 8                                  # step a3 joins the cluster's launch for up to 8 KV heads
         assert g.ctx.tf_get_status()[1]["launches"] == launches + (1 if one_launch else 2)
         for got, want in zip((g.score, g.keep, g.idx, g.nk, g.theta), two):
             assert torch.equal(got.view(torch.int32) if got.dtype == torch.float32 else got,
