@@ -55,7 +55,8 @@ struct TcParams {
     DevStatus* status;
     int compact;          // 1: K / V hold the retained tokens only, entry c = token kept_idx[c] (TF_KV_RETAINED)
     int n_row_blocks;     // CTAs per (batch, query head)
-    int heads_fastest;    // CTA order: 1 = all heads of the heaviest row block first, 0 = all row blocks of a head together
+    int bh_group;         // CTA order: (batch, head) pairs are taken in groups of this many; within a group all of the
+                          // heaviest row block first.  1 = all row blocks of a head together, n_bh = heaviest first over all heads
     int first_pair;       // row block the first CTA of a head takes: the last one expected to hold retained rows
     long long wait_cycles;   // budget of one mbarrier wait
 };
@@ -76,6 +77,20 @@ template <bool kSplit> struct Cfg {
     static constexpr int kOffBar = kOffRing + kStages * kTileBytes;
     static constexpr int kSmemBytes = kOffBar + 256 + 1024;   // barriers + alignment slack
 };
+
+// CTAs start in index order.  Row blocks of a head differ in length by the causal triangle, so the heaviest should
+// go first, over as many heads as possible (the grid then ends with short CTAs from many heads, which fill the SMs
+// evenly); but the CTAs that run at the same time should find K and V in L2, which the row blocks of one head do (they
+// read nearly the same keys) and those of different heads do not.  So the (batch, head) pairs are taken in groups whose
+// K and V fit the L2 budget, and inside a group the order is: heaviest row block of every head, next row block, ...
+__device__ __forceinline__ void cta_work_item(const TcParams& p, int& rb, int& bh) {
+    const int n_bh = (int)(gridDim.x / (unsigned)p.n_row_blocks);
+    const int per_group = p.bh_group * p.n_row_blocks;
+    const int g = (int)blockIdx.x / per_group, within = (int)blockIdx.x - g * per_group;
+    const int g_size = min(p.bh_group, n_bh - g * p.bh_group);     // the last group may be smaller
+    rb = within / g_size;
+    bh = g * p.bh_group + within % g_size;
+}
 
 // bounded wait; after the first expiry in this CTA nobody waits any more
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget_cycles,
@@ -243,12 +258,8 @@ attention_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap mapK, 
     __syncwarp();
     if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     grid_dependency_wait();   // kept_idx / n_kept come from the kernel before this one
-    // CTAs start in index order.  Row blocks of a head differ in length by the causal triangle, so the
-    // heaviest go first; with few CTAs per SM that has to hold across heads (heads_fastest), while a
-    // large problem keeps the row blocks of one head together so that they find its K/V in L2.
-    const int n_bh = (int)(gridDim.x / (unsigned)p.n_row_blocks);
-    const int rb = p.heads_fastest ? (int)blockIdx.x / n_bh : (int)blockIdx.x % p.n_row_blocks;
-    const int bh = p.heads_fastest ? (int)blockIdx.x % n_bh : (int)blockIdx.x / p.n_row_blocks;
+    int rb, bh;
+    cta_work_item(p, rb, bh);
     // Row blocks are taken from the heaviest expected one (the last with retained rows, a host-side estimate) down to
     // block 0, then the blocks above the estimate, which are normally empty: CTAs with nothing to do start last
     // instead of delaying the first wave of real work.  Any estimate gives a one-to-one assignment.
@@ -625,9 +636,8 @@ attention_tc_single_kernel(const TcParams p, const __grid_constant__ CUtensorMap
     __syncwarp();
     if (warp == kMmaWarp1) tmem_alloc(smem_u32(tmem_slot), kTmemCols1);
     grid_dependency_wait();   // kept_idx / n_kept come from the kernel before this one
-    const int n_bh = (int)(gridDim.x / (unsigned)p.n_row_blocks);
-    const int rb = p.heads_fastest ? (int)blockIdx.x / n_bh : (int)blockIdx.x % p.n_row_blocks;
-    const int bh = p.heads_fastest ? (int)blockIdx.x % n_bh : (int)blockIdx.x / p.n_row_blocks;
+    int rb, bh;
+    cta_work_item(p, rb, bh);
     int blk = p.first_pair - rb;          // heaviest expected row block first, blocks expected to be empty last
     if (blk < 0) blk += p.n_row_blocks;
     const int qh = bh % p.Hq, b = bh / p.Hq;
@@ -963,9 +973,22 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         const long long blocks = (std::max<long long>(kept_est, 1) + rows_per_cta - 1) / rows_per_cta;
         tp.first_pair = (int)std::min<long long>(std::max<long long>(blocks - 1, 0), tp.n_row_blocks - 1);
     }
-    const double kv_bytes = 2.0 * s.batch * s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
-    tp.heads_fastest = (kv_bytes <= 48e6 || ctas_shared < 6.0 * sms) ? 1 : 0;   // K and V stay in L2, or balance matters more
-    const long long n_ctas = (long long)tp.n_row_blocks * (heads ? s.n_q_heads / (2 * hpt) : s.n_q_heads) * s.batch;
+    const long long n_bh = (long long)(heads ? s.n_q_heads / (2 * hpt) : s.n_q_heads) * s.batch;
+    const long long n_ctas = (long long)tp.n_row_blocks * n_bh;
+    {
+        // Groups of (batch, head) pairs.  Heaviest-first over ALL heads balances best and costs nothing while all of K
+        // and V stays in L2 (c4: 555 -> 526 us).  Once the K and V of the heads that run together exceed L2, every CTA
+        // streams its keys from HBM (3.9 KB per MFLOP of tile products): in short loops the balance still wins
+        // (c3: 405 -> 372 us), under the power cap of a long run the HBM traffic lowers the clock and loses
+        // (425 -> 445 us), and groups sized to fit L2 (32 heads on c3) came out within the noise of one head at a
+        // time; a window makes the row blocks equally long, so there is nothing to balance (c5: any larger group
+        // measured 2-12 % slower).  So: all heads when K and V fit kL2Budget or the grid has only a few CTAs per SM,
+        // else one pair at a time.
+        constexpr double kL2Budget = 72e6;
+        const double kv_all = 2.0 * s.batch * (double)s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
+        const long long g = (kv_all <= kL2Budget || ctas_shared < 6.0 * sms) ? n_bh : 1;
+        tp.bh_group = (int)std::min<long long>(std::max<long long>(g, 1), std::max<long long>(n_bh, 1));
+    }
     if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
     cudaError_t e;
     if (single) e = launch_dependent(attention_tc_single_kernel, dim3((unsigned)n_ctas), dim3(kThreads1), kSmemBytes1, st, tp, mapK, mapV);
