@@ -980,13 +980,19 @@ cudaError_t launch_attention_tc(tf_ctx* ctx, const tf_shape& s, const tf_filter_
         // and V stays in L2 (c4: 555 -> 526 us).  Once the K and V of the heads that run together exceed L2, every CTA
         // streams its keys from HBM (3.9 KB per MFLOP of tile products): in short loops the balance still wins
         // (c3: 405 -> 372 us), under the power cap of a long run the HBM traffic lowers the clock and loses
-        // (425 -> 445 us), and groups sized to fit L2 (32 heads on c3) came out within the noise of one head at a
-        // time; a window makes the row blocks equally long, so there is nothing to balance (c5: any larger group
-        // measured 2-12 % slower).  So: all heads when K and V fit kL2Budget or the grid has only a few CTAs per SM,
-        // else one pair at a time.
+        // (425 -> 445 us).  So a group is as many pairs as keep their K and V within kL2Budget, in equal groups
+        // (c3: 5 groups of 32 heads, 438 -> 422 us in long loops, 430 -> 397 in short ones).  A window makes the row
+        // blocks equally long, so there is nothing to balance and the row blocks of a pair stay together (c5: every
+        // larger group measured 2-12 % slower).  A grid of a few CTAs per SM is balanced over all heads whatever the size.
         constexpr double kL2Budget = 72e6;
         const double kv_all = 2.0 * s.batch * (double)s.seq * s.n_kv_heads * kHeadDim * sizeof(__nv_bfloat16);
-        const long long g = (kv_all <= kL2Budget || ctas_shared < 6.0 * sms) ? n_bh : 1;
+        const double kv_per_bh = kv_all / (double)std::max<long long>(n_bh, 1);
+        const bool windowed = s.window > 0 && (long long)s.window + 1024 < s.seq;
+        long long g = windowed ? 1 : std::max<long long>((long long)(kL2Budget / kv_per_bh), 1);
+        if (kv_all <= kL2Budget || ctas_shared < 6.0 * sms) g = n_bh;
+        g = std::min<long long>(g, std::max<long long>(n_bh, 1));
+        const long long n_groups = (std::max<long long>(n_bh, 1) + g - 1) / g;      // equal groups, not a small last one
+        g = (std::max<long long>(n_bh, 1) + n_groups - 1) / n_groups;
         tp.bh_group = (int)std::min<long long>(std::max<long long>(g, 1), std::max<long long>(n_bh, 1));
     }
     if (n_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
