@@ -431,6 +431,37 @@ def test_pruned_attention_nothing_kept_and_everything_kept(path):
     g.close()
 
 
+def test_pruned_attention_head_groups_of_unequal_size():
+    """A shape whose K and V exceed the L2 budget of the CTA order and whose (batch, head) pairs do not divide into
+    equal groups (2 x 57 heads of 4096 tokens: groups of 29, 29, 29 and 27): every row block of every head must still be
+    served exactly once.  Sampled rows against the oracle, the rest through properties that hold at any size."""
+    B, S, H = 2, 4096, 57
+    q, k, v = _qkv(B, S, H, H, torch.bfloat16, seed=57)
+    rng = np.random.default_rng(57)
+    score = rng.normal(0.2, 0.2, (B, S))
+    ref = oracle.select(score, 0.5, 4)
+    g = Gpu(q, k, v, prune_ratio=0.5, warmup_tokens=4)
+    g.ctx.tf_set_attention_path(2)
+    idx, nk = torch.from_numpy(ref["kept_idx"]).to(DEV), torch.from_numpy(ref["n_kept"]).to(DEV)
+    g.ctx.tf_pruned_attention(g.shape, g.params, q, k, v, idx, nk, g.O)
+    g.status_ok()
+    assert g.ctx.tf_last_kernels()[1] == tfb.TF_KERNEL_ATTN_TC_SHARED
+    keep_d = torch.from_numpy(ref["keep_mask"]).to(DEV).bool()
+    assert bool((g.O[~keep_d] == 0).all()) and bool(torch.isfinite(g.O[keep_d]).all())
+    assert bool((g.O[keep_d].float().abs().amax(dim=-1) > 0).all())          # every retained row of every head was written
+    n = 1500
+    bs = rng.integers(B, size=n)
+    ts = np.array([ref["kept_idx"][b, rng.integers(ref["n_kept"][b])] for b in bs])
+    hs = np.concatenate([np.arange(H), rng.integers(H, size=n - H)])          # every head at least once
+    rows = np.stack([bs, ts, hs], 1).astype(np.int32)
+    qn, kn, vn = q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy()
+    want = oracle.attention_rows(qn, kn, vn, ref["keep_mask"], rows)
+    got = g.O[rows[:, 0], rows[:, 1], rows[:, 2]].float().cpu().numpy().astype(np.float64)
+    scale = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
+    assert float((np.abs(got - want) / scale).max()) < ATTN_TOL[torch.bfloat16]
+    g.close()
+
+
 @pytest.mark.parametrize("tensor_cores", [2, 3, 4, 5, 6])
 @pytest.mark.parametrize("claimed_ratio", [0.0, 0.9])
 def test_pruned_attention_with_a_retained_list_the_ratio_does_not_predict(tensor_cores, claimed_ratio):
