@@ -30,6 +30,17 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// four consecutive elements (16 bytes of fp32, 8 bytes of bf16; the caller's offset is a multiple of four elements)
+__device__ __forceinline__ void load4(const float* p, float (&f)[4]) {
+    const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&f)[4]) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+
 template <typename T>
 __device__ __forceinline__ void zero_rows(T* Ob, const Strides3& os, int t_lo, int t_hi, int lane) {
     for (int t = t_lo; t < t_hi; ++t) {
@@ -80,8 +91,9 @@ __global__ void __launch_bounds__(kSimtWarps * 32) attention_simt_kernel(const A
         if (j <= j_hi) {
             const T* krow = Kb + (long long)tok * p.ks.t;
             float d0 = 0.f, d1 = 0.f;
-#pragma unroll 4
-            for (int v = 0; v < NVEC; ++v) {
+#pragma unroll 8
+            for (int v = 0; v < NVEC; ++v) {   // eight 16-byte loads in flight per lane: the warp is alone on its row, so
+                                               // memory-level parallelism has to come from inside it
                 float f[EPV];
                 Elem<T>::unpack(ldg16(krow + v * EPV), f);
                 const float* qq = &q_s[warp][v * EPV];
@@ -97,12 +109,23 @@ __global__ void __launch_bounds__(kSimtWarps * 32) attention_simt_kernel(const A
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[i] *= corr;
         const int n_here = min(32, j_hi - j0 + 1);
-        for (int jj = 0; jj < n_here; ++jj) {
-            const float pw = __shfl_sync(0xffffffffu, pj, jj);
-            const int vt = __shfl_sync(0xffffffffu, tok, jj);
-            const T* vrow = Vb + (long long)vt * p.vs.t + lane * 4;
+        // same order of additions as a plain loop over the block's keys; the value rows of eight keys are requested
+        // together (loads first, products after), not one round trip to memory per key
+        for (int jj0 = 0; jj0 < n_here; jj0 += 8) {
+            float vv[8][4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[i] = fmaf(pw, to_f<T>(vrow[i]), acc[i]);
+            for (int u = 0; u < 8; ++u) {
+                const int vt = __shfl_sync(0xffffffffu, tok, jj0 + u);
+                if (jj0 + u < n_here) load4(Vb + (long long)vt * p.vs.t + lane * 4, vv[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float pw = __shfl_sync(0xffffffffu, pj, jj0 + u);
+                if (jj0 + u < n_here) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[i] = fmaf(pw, vv[u][i], acc[i]);
+                }
+            }
         }
         m = m_new;
     }
