@@ -13,7 +13,8 @@
 //   * step a4, RATIO mode: the same 4-pass, 8-bit MSB-first radix select over order-preserving keys as the
 //     one-CTA kernel.  Each CTA histograms its own candidates; after a cluster barrier every CTA adds up the
 //     cluster's histograms through distributed shared memory and takes the same decision (two histogram buffers
-//     alternate, so one cluster barrier per pass is enough);
+//     alternate, so one cluster barrier per pass is enough); once at most 32 candidates share the prefix they are
+//     appended to a list in CTA 0's shared memory and every CTA ranks them there instead of further passes;
 //   * ranks in index order (which of the tokens that tie with the P-th key go, and where a retained token lands in
 //     kept_idx) are a CTA-local scan plus the totals of the CTAs before it in the cluster, again through
 //     distributed shared memory.
